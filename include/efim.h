@@ -1,0 +1,159 @@
+/*
+ * efim.h - C ABI of the EFIM per-turn GPU path (NVIDIA B200, sm_100a).
+ *
+ * EFIM (Sec. 1; Sec. 2.2, Fig. 3) rewrites an infilling prompt from
+ * `<P>prefix+inc<S>suffix<M>` to `<P>prefix<S>suffix<M>inc`.  The keys and
+ * values of `<P>prefix<S>suffix<M>` (C tokens) then stay valid in the paged KV
+ * cache from one turn to the next; each turn only has to
+ *   1. rotate the N new `inc` tokens' q/k by their positions C..C+N-1 and store
+ *      k/v into the cache pages                       -> efim_kv_append
+ *   2. attend the N new queries causally over the C cached and N new keys
+ *                                                     -> efim_append_prefill_attn
+ *   3. decode the generated middle one token at a time -> efim_decode_attn
+ * The paper changes nothing in the model (Sec. 3), so 2 and 3 are standard
+ * softmax attention, o = sum_j softmax_j(scale * q.k_j) v_j.
+ *
+ * Conventions for every entry point
+ *   - Pointers named d_* are DEVICE pointers, h_* are HOST pointers.  The caller
+ *     owns all memory and the stream; the library allocates no device memory,
+ *     keeps no state between calls and never synchronises the device.
+ *   - `stream` is a cudaStream_t passed as void* (NULL = default stream).  All
+ *     work is enqueued on it; results are ready when the stream reaches that point.
+ *   - bf16 tensors are raw 16-bit patterns.  Packed layouts, innermost last:
+ *       q / out      [total_new_tokens][num_q_heads][head_dim]   bf16
+ *       k_new/v_new  [total_new_tokens][num_kv_heads][head_dim]  bf16
+ *       pools        [num_pages][num_kv_heads][page_size][head_dim] bf16 (K and V separate)
+ *       block table  [batch][max_pages_per_seq] int32: token p of sequence s lives
+ *                    in page block_table[s][p / page_size], slot p % page_size.
+ *     Sequence s owns rows q_indptr[s] .. q_indptr[s+1]-1 of the packed tensors.
+ *   - Grouped-query map: q head h reads kv head h / (num_q_heads / num_kv_heads).
+ *   - Errors the host can see (null pointers, unsupported shapes, workspace too
+ *     small) are returned before anything is launched.  Errors only the device can
+ *     see are OR-ed into *d_status (EFIM_DEV_* bits) if d_status is not NULL, and the
+ *     offending access is skipped; the kernels never trap.
+ *   - Supported: page_size 16; head_dim 64 or 128; num_q_heads a multiple of
+ *     num_kv_heads; base pointers 16-byte aligned (pools 128-byte aligned).
+ */
+#ifndef EFIM_H_
+#define EFIM_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum {
+  EFIM_OK = 0,
+  EFIM_ERR_INVALID_ARG = 1,   /* null pointer, negative size, H_q % H_kv != 0, bad alignment */
+  EFIM_ERR_UNSUPPORTED = 2,   /* head_dim / page_size outside the supported set            */
+  EFIM_ERR_OUT_OF_RANGE = 3,  /* a host-visible length exceeds max_pages_per_seq*page_size  */
+  EFIM_ERR_WORKSPACE = 4,     /* workspace_bytes smaller than the *_workspace_bytes() answer */
+  EFIM_ERR_CUDA = 5,          /* a CUDA runtime/driver call failed (launch, copy, tensor map) */
+  EFIM_ERR_TIMEOUT = 6        /* reserved: reported through d_status by bounded device waits */
+} efim_status;
+
+/* Bits OR-ed into *d_status by kernels. */
+#define EFIM_DEV_BAD_PAGE      0x1   /* block-table entry outside [0, num_pages)           */
+#define EFIM_DEV_BAD_POSITION  0x2   /* token position >= rope max_position, or beyond table */
+#define EFIM_DEV_TIMEOUT       0x4   /* a bounded wait inside a kernel expired               */
+
+const char* efim_strerror(efim_status s);
+int efim_version(void);
+
+/* Paged KV cache of ONE layer. */
+typedef struct {
+  void* d_k_pool;            /* bf16 [num_pages][num_kv_heads][page_size][head_dim] */
+  void* d_v_pool;            /* same shape                                         */
+  int32_t num_pages;
+  int32_t page_size;         /* 16 */
+  int32_t num_q_heads;
+  int32_t num_kv_heads;
+  int32_t head_dim;          /* 64 or 128 */
+} efim_cache_desc;
+
+/* Ragged batch of one turn: sequence s has cached_len[s] tokens already in the
+ * cache (`<P>prefix<S>suffix<M>`) and new_len[s] new tokens (`inc`). */
+typedef struct {
+  int32_t batch;
+  int32_t max_pages_per_seq;
+  int32_t total_new_tokens;          /* = q_indptr[batch]                             */
+  const int32_t* d_cached_len;       /* [batch]                                       */
+  const int32_t* d_new_len;          /* [batch]                                       */
+  const int32_t* d_q_indptr;         /* [batch+1], exclusive prefix sum of new_len    */
+  const int32_t* d_block_table;      /* [batch][max_pages_per_seq]                    */
+  const int32_t* h_cached_len;       /* host mirrors, read during the call (planning) */
+  const int32_t* h_new_len;
+} efim_batch_desc;
+
+/* Rotary embedding.  d_cos_sin row p holds cos(p*theta_f), f = 0..D/2-1, then
+ * sin(p*theta_f), f = 0..D/2-1, theta_f = base^(-2f/D).  Pair (f, f+D/2) is
+ * rotated, or (2f, 2f+1) when interleaved != 0.  d_cos_sin == NULL disables the
+ * rotation (k is stored as given, q untouched). */
+typedef struct {
+  const float* d_cos_sin;    /* fp32 [max_position][head_dim] */
+  int32_t max_position;
+  int32_t interleaved;
+} efim_rope_desc;
+
+/* Fill a HOST table for efim_rope_desc (computed in double, rounded to float).
+ * h_out: [max_position][head_dim] floats owned by the caller. */
+efim_status efim_rope_table_build(double base, int32_t head_dim, int32_t max_position, float* h_out);
+
+/*
+ * Step 1 (EFIM Sec. 1: only `inc` is new; its k/v join the cache after
+ * `<P>prefix<S>suffix<M>`).  For new token i of sequence s, position
+ * p = cached_len[s] + i: q and k are rotated by p (fp32 math, one bf16
+ * round-to-nearest-even), q is rewritten in place, k (rotated) and v (as is) are
+ * stored at page block_table[s][p/page_size], slot p%page_size, all kv heads.
+ * d_q may be NULL (only k/v are processed).  Sequences must not share a page that
+ * is written.  A bad page id or position sets a bit in *d_status and skips that token.
+ */
+efim_status efim_kv_append(const efim_cache_desc* cache, const efim_batch_desc* batch,
+                           const efim_rope_desc* rope,
+                           void* d_q, const void* d_k_new, const void* d_v_new,
+                           int32_t* d_status, void* stream);
+
+/*
+ * Step 2 (EFIM Sec. 1, Sec. 2.2: prefix and suffix KV are cache hits, so the
+ * prefill that remains is the `inc` tokens attending over everything before
+ * them).  The new tokens' k/v must already be in the pages (efim_kv_append).
+ * New token i of sequence s (position C+i) sees keys j <= C+i:
+ *   out[t,h,:] = sum_j softmax_j(sm_scale * q[t,h,:].k[j,h/G,:]) v[j,h/G,:]
+ *   lse[t,h]   = log sum_j exp(sm_scale * q.k_j)         (natural log; optional)
+ * bf16 operands, fp32 accumulation and softmax, bf16 output.
+ * sm_scale <= 0 selects 1/sqrt(head_dim).  Sequences with new_len 0 are skipped.
+ * The host mirrors h_cached_len/h_new_len are read during the call to build the
+ * work list, which is copied into the workspace on `stream`.
+ * Workspace: at least efim_prefill_workspace_bytes() bytes, 256-byte aligned,
+ * exclusively this call's until the stream has passed it.
+ */
+size_t efim_prefill_workspace_bytes(const efim_cache_desc* cache, const efim_batch_desc* batch);
+efim_status efim_append_prefill_attn(const efim_cache_desc* cache, const efim_batch_desc* batch,
+                                     const void* d_q, void* d_out, float* d_lse, float sm_scale,
+                                     void* d_workspace, size_t workspace_bytes,
+                                     int32_t* d_status, void* stream);
+
+/*
+ * Step 3 (decode of the generated middle, EFIM Sec. 2.2 / Fig. 4): one query
+ * token per sequence over keys [0, ctx_len[s]) (ctx_len counts the token just
+ * appended).  The key range is cut into fixed-length chunks; each chunk yields a
+ * partial (o_c, lse_c) in the workspace and a second kernel merges them:
+ *   lse = log sum_c exp(lse_c),  o = sum_c exp(lse_c - lse) o_c.
+ * max_ctx_len is an upper bound on every ctx_len[s] (<= 0: max_pages_per_seq *
+ * page_size); it fixes the chunking, so no host copy of the lengths is needed.
+ * ctx_len[s] == 0 gives out = 0, lse = -inf.
+ */
+size_t efim_decode_workspace_bytes(const efim_cache_desc* cache, int32_t batch, int32_t max_ctx_len);
+efim_status efim_decode_attn(const efim_cache_desc* cache, int32_t batch,
+                             const int32_t* d_ctx_len, int32_t max_ctx_len,
+                             const int32_t* d_block_table, int32_t max_pages_per_seq,
+                             const void* d_q, void* d_out, float* d_lse, float sm_scale,
+                             void* d_workspace, size_t workspace_bytes,
+                             int32_t* d_status, void* stream);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* EFIM_H_ */

@@ -1,0 +1,64 @@
+// Shared host/device helpers for the EFIM kernels (sm_100a).
+#pragma once
+#include <cuda_runtime.h>
+#include <cuda_bf16.h>
+#include <stdint.h>
+#include "efim.h"
+
+#define EFIM_CUDA_TRY(expr)                          \
+  do {                                               \
+    cudaError_t e__ = (expr);                        \
+    if (e__ != cudaSuccess) return EFIM_ERR_CUDA;    \
+  } while (0)
+
+namespace efim {
+
+// Validation shared by every entry point: shapes the kernels are built for.
+inline efim_status check_cache(const efim_cache_desc* c) {
+  if (!c || !c->d_k_pool || !c->d_v_pool) return EFIM_ERR_INVALID_ARG;
+  if (c->num_pages <= 0 || c->num_q_heads <= 0 || c->num_kv_heads <= 0) return EFIM_ERR_INVALID_ARG;
+  if (c->num_q_heads % c->num_kv_heads != 0) return EFIM_ERR_INVALID_ARG;
+  if (c->page_size != 16) return EFIM_ERR_UNSUPPORTED;
+  if (c->head_dim != 64 && c->head_dim != 128) return EFIM_ERR_UNSUPPORTED;
+  if ((reinterpret_cast<uintptr_t>(c->d_k_pool) & 127) || (reinterpret_cast<uintptr_t>(c->d_v_pool) & 127))
+    return EFIM_ERR_INVALID_ARG;
+  return EFIM_OK;
+}
+
+inline efim_status check_batch(const efim_cache_desc* c, const efim_batch_desc* b, bool need_host) {
+  if (!b) return EFIM_ERR_INVALID_ARG;
+  if (b->batch < 0 || b->total_new_tokens < 0 || b->max_pages_per_seq <= 0) return EFIM_ERR_INVALID_ARG;
+  if (b->batch == 0) return EFIM_OK;
+  if (!b->d_cached_len || !b->d_new_len || !b->d_q_indptr || !b->d_block_table) return EFIM_ERR_INVALID_ARG;
+  if (need_host) {
+    if (!b->h_cached_len || !b->h_new_len) return EFIM_ERR_INVALID_ARG;
+    long long total = 0;
+    const long long cap = (long long)b->max_pages_per_seq * c->page_size;
+    for (int s = 0; s < b->batch; ++s) {
+      if (b->h_cached_len[s] < 0 || b->h_new_len[s] < 0) return EFIM_ERR_INVALID_ARG;
+      if ((long long)b->h_cached_len[s] + b->h_new_len[s] > cap) return EFIM_ERR_OUT_OF_RANGE;
+      total += b->h_new_len[s];
+    }
+    if (total != b->total_new_tokens) return EFIM_ERR_INVALID_ARG;
+  }
+  return EFIM_OK;
+}
+
+__device__ __forceinline__ float bf16lo(uint32_t w) { return __uint_as_float(w << 16); }
+__device__ __forceinline__ float bf16hi(uint32_t w) { return __uint_as_float(w & 0xffff0000u); }
+
+// two floats -> packed bf16x2 (round to nearest even); lo lands in the low half
+__device__ __forceinline__ uint32_t pack_bf16x2(float lo, float hi) {
+  uint32_t r;
+  asm("cvt.rn.bf16x2.f32 %0, %1, %2;" : "=r"(r) : "f"(hi), "f"(lo));
+  return r;
+}
+
+__device__ __forceinline__ uint4 ldg_stream(const void* p) {
+  uint4 v;
+  asm volatile("ld.global.nc.L1::no_allocate.v4.u32 {%0,%1,%2,%3}, [%4];"
+               : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "l"(p));
+  return v;
+}
+
+}  // namespace efim

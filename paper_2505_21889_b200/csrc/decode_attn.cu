@@ -1,0 +1,377 @@
+// efim_decode_attn: split-KV paged decode attention with a log-sum-exp merge
+// (decode of the generated middle, EFIM Sec. 2.2 / Fig. 4).  Bandwidth-bound:
+// every K/V byte of the visible context is read once with 128-bit loads, the dot
+// products run on fp32 FMAs, the reductions on warp shuffles; no tensor cores.
+//
+// One CTA = (query row, kv head [x group tile], key chunk).  Each of its 4 warps
+// walks whole pages (16 tokens) round-robin.  Inside a warp D/8 lanes share one
+// token row (16 bytes each), so 32/(D/8) tokens are in flight per load.
+#include "decode_attn.cuh"
+
+namespace efim {
+
+// Sum x[0..N) across the `LPT` lanes of a token group, leaving N/LPT sums per lane.
+// Round with lane-bit `off`: lanes with the bit clear keep the lower half of the
+// values and receive the partner's lower half; the others the upper half.  After
+// all rounds lane j holds the values whose index has, from the top bit down, the
+// bits of j; the remaining low index bits enumerate the values it keeps.
+template <int N, int LPT>
+__device__ __forceinline__ void transposed_reduce(float* x, int j) {
+  int n = N;
+#pragma unroll
+  for (int off = LPT / 2; off >= 1; off >>= 1) {
+    const int half = n / 2;
+    const bool up = (j & off) != 0;
+#pragma unroll
+    for (int i = 0; i < N / 2; ++i) {
+      if (i < half) {
+        const float send = up ? x[i] : x[i + half];
+        const float keep = up ? x[i + half] : x[i];
+        x[i] = keep + __shfl_xor_sync(0xffffffffu, send, off);
+      }
+    }
+    n = half;
+  }
+}
+
+template <int D, int GT>
+__global__ void __launch_bounds__(128) decode_splitkv_kernel(const DecodeParams p) {
+  constexpr int LPT = D / 8;            // lanes sharing one token row
+  constexpr int TPS = 32 / LPT;         // tokens per warp-wide load
+  constexpr int STEPS = 16 / TPS;       // loads per page
+  constexpr int GP = (GT + 1) & ~1;     // heads padded to even
+  constexpr int NV = STEPS * GP;        // partial dot products per lane per page
+  constexpr int NF = GP / 2;            // finished scores per lane per page
+  static_assert(NV / LPT == NF, "reduction leaves GP/2 values per lane");
+
+  __shared__ float s_p[4][16][GP];      // per warp: probabilities of the current page
+  __shared__ float s_m[4][GP], s_l[4][GP];
+  __shared__ float s_o[4][GT][D];
+
+  const int r = blockIdx.x;
+  const int G = p.Hq / p.Hkv;
+  const int gsplit = (G + GT - 1) / GT;
+  const int kvh = blockIdx.y / gsplit;
+  const int g0 = (blockIdx.y % gsplit) * GT;
+  const int ng = min(GT, G - g0);
+  const int c = blockIdx.z;
+  const int len = __ldg(p.row_len + r);
+  const int begin = c * p.chunk_tokens;
+  const int head0 = kvh * G + g0;
+  const int tid = threadIdx.x;
+  if (begin >= len) {
+    // nothing visible in this chunk; a row without any key still gets a defined result
+    if (len <= 0 && c == 0 && p.n_chunks == 1) {
+      for (int i = tid; i < ng * D; i += 128) p.out[((size_t)r * p.Hq + head0) * D + i] = 0;
+      if (p.lse && tid < ng) p.lse[(size_t)r * p.Hq + head0 + tid] = -INFINITY;
+    }
+    return;
+  }
+  const int end = min(len, begin + p.chunk_tokens);
+  const int seq = p.row_seq ? __ldg(p.row_seq + r) : r;
+  const int lane = tid & 31, warp = tid >> 5;
+  const int j = lane % LPT, tg = lane / LPT;
+
+  float q[GT][8];
+#pragma unroll
+  for (int g = 0; g < GT; ++g) {
+    if (g < ng) {
+      const uint4 w = __ldg(reinterpret_cast<const uint4*>(p.q + ((size_t)r * p.Hq + head0 + g) * D) + j);
+      const uint32_t* u = reinterpret_cast<const uint32_t*>(&w);
+#pragma unroll
+      for (int e = 0; e < 4; ++e) {
+        q[g][2 * e] = bf16lo(u[e]) * p.scale_log2;
+        q[g][2 * e + 1] = bf16hi(u[e]) * p.scale_log2;
+      }
+    } else {
+#pragma unroll
+      for (int e = 0; e < 8; ++e) q[g][e] = 0.f;
+    }
+  }
+  float o[GT][8];
+#pragma unroll
+  for (int g = 0; g < GT; ++g)
+#pragma unroll
+    for (int e = 0; e < 8; ++e) o[g][e] = 0.f;
+  float m_run[GP], l_part[NF];
+#pragma unroll
+  for (int g = 0; g < GP; ++g) m_run[g] = -INFINITY;
+#pragma unroll
+  for (int i = 0; i < NF; ++i) l_part[i] = 0.f;
+
+  const int32_t* bt = p.block_table + (size_t)seq * p.max_pages_per_seq;
+  const int odd = j & 1;
+  const int st_mine = j >> 1;                   // step whose scores this lane ends up with
+
+  for (int pg = (begin >> 4) + warp; (pg << 4) < end; pg += 4) {
+    const int page = __ldg(bt + pg);
+    if (page < 0 || page >= p.num_pages) {      // warp-uniform
+      if (lane == 0 && p.status) atomicOr(p.status, EFIM_DEV_BAD_PAGE);
+      continue;
+    }
+    const size_t base = (((size_t)page * p.Hkv + kvh) * 16 + tg) * D + j * 8;
+    uint4 kreg[STEPS], vreg[STEPS];
+#pragma unroll
+    for (int st = 0; st < STEPS; ++st) kreg[st] = ldg_stream(p.k_pool + base + (size_t)st * TPS * D);
+#pragma unroll
+    for (int st = 0; st < STEPS; ++st) vreg[st] = ldg_stream(p.v_pool + base + (size_t)st * TPS * D);
+
+    // ---- scores: partial dot products over this lane's 8 dims, then the cross-lane sum
+    float x[NV];
+#pragma unroll
+    for (int st = 0; st < STEPS; ++st) {
+      const uint32_t* u = reinterpret_cast<const uint32_t*>(&kreg[st]);
+      float kf[8];
+#pragma unroll
+      for (int e = 0; e < 4; ++e) { kf[2 * e] = bf16lo(u[e]); kf[2 * e + 1] = bf16hi(u[e]); }
+#pragma unroll
+      for (int g = 0; g < GP; ++g) {
+        float acc = 0.f;
+        if (g < GT) {
+#pragma unroll
+          for (int e = 0; e < 8; ++e) acc = fmaf(q[g][e], kf[e], acc);
+        }
+        x[st * GP + g] = acc;
+      }
+    }
+    transposed_reduce<NV, LPT>(x, j);
+    // lane j now holds, for token (st_mine*TPS + tg) of the page, heads odd*NF + i
+    const int tok_in_page = st_mine * TPS + tg;
+    const bool visible = (pg << 4) + tok_in_page < end;
+    float sc[NF], mx[NF];
+#pragma unroll
+    for (int i = 0; i < NF; ++i) { sc[i] = visible ? x[i] : -INFINITY; mx[i] = sc[i]; }
+#pragma unroll
+    for (int off = 2; off < 32; off <<= 1)
+#pragma unroll
+      for (int i = 0; i < NF; ++i) mx[i] = fmaxf(mx[i], __shfl_xor_sync(0xffffffffu, mx[i], off));
+    float alpha[GP], mine[NF], alpha_mine[NF];
+#pragma unroll
+    for (int i = 0; i < NF; ++i) {
+      const float other = __shfl_xor_sync(0xffffffffu, mx[i], 1);
+      const float m_lo = odd ? other : mx[i];       // head i
+      const float m_hi = odd ? mx[i] : other;       // head NF + i
+      const float n_lo = fmaxf(m_run[i], m_lo), n_hi = fmaxf(m_run[NF + i], m_hi);
+      alpha[i] = exp2f(m_run[i] - n_lo);
+      alpha[NF + i] = exp2f(m_run[NF + i] - n_hi);
+      m_run[i] = n_lo;
+      m_run[NF + i] = n_hi;
+      mine[i] = odd ? n_hi : n_lo;
+      alpha_mine[i] = odd ? alpha[NF + i] : alpha[i];
+    }
+#pragma unroll
+    for (int i = 0; i < NF; ++i) {
+      const float pr = exp2f(sc[i] - mine[i]);      // masked: exp2(-inf) = 0
+      l_part[i] = fmaf(l_part[i], alpha_mine[i], pr);
+      s_p[warp][tok_in_page][odd * NF + i] = pr;
+    }
+    __syncwarp();
+    // ---- values
+#pragma unroll
+    for (int g = 0; g < GT; ++g)
+#pragma unroll
+      for (int e = 0; e < 8; ++e) o[g][e] *= alpha[g];
+#pragma unroll
+    for (int st = 0; st < STEPS; ++st) {
+      const int tp = st * TPS + tg;
+      if ((pg << 4) + tp < end) {                   // never touch slots past the context
+        const uint32_t* u = reinterpret_cast<const uint32_t*>(&vreg[st]);
+        float vf[8];
+#pragma unroll
+        for (int e = 0; e < 4; ++e) { vf[2 * e] = bf16lo(u[e]); vf[2 * e + 1] = bf16hi(u[e]); }
+#pragma unroll
+        for (int g = 0; g < GT; ++g) {
+          const float pr = s_p[warp][tp][g];
+#pragma unroll
+          for (int e = 0; e < 8; ++e) o[g][e] = fmaf(pr, vf[e], o[g][e]);
+        }
+      }
+    }
+    __syncwarp();
+  }
+
+  // ---- fold the token groups of the warp, then the 4 warps
+#pragma unroll
+  for (int off = LPT; off < 32; off <<= 1)
+#pragma unroll
+    for (int g = 0; g < GT; ++g)
+#pragma unroll
+      for (int e = 0; e < 8; ++e) o[g][e] += __shfl_xor_sync(0xffffffffu, o[g][e], off);
+#pragma unroll
+  for (int off = 2; off < 32; off <<= 1)
+#pragma unroll
+    for (int i = 0; i < NF; ++i) l_part[i] += __shfl_xor_sync(0xffffffffu, l_part[i], off);
+  if (lane < 2) {
+#pragma unroll
+    for (int i = 0; i < NF; ++i) s_l[warp][lane * NF + i] = l_part[i];
+  }
+  if (lane == 0) {
+#pragma unroll
+    for (int g = 0; g < GP; ++g) s_m[warp][g] = m_run[g];
+  }
+  if (tg == 0) {
+#pragma unroll
+    for (int g = 0; g < GT; ++g)
+#pragma unroll
+      for (int e = 0; e < 8; ++e) s_o[warp][g][j * 8 + e] = o[g][e];
+  }
+  __syncthreads();
+  for (int idx = tid; idx < ng * D; idx += 128) {
+    const int g = idx / D, d = idx % D;
+    float M = fmaxf(fmaxf(s_m[0][g], s_m[1][g]), fmaxf(s_m[2][g], s_m[3][g]));   // warp 0 always has a page
+    float L = 0.f, O = 0.f;
+#pragma unroll
+    for (int w = 0; w < 4; ++w) {
+      const float sc = exp2f(s_m[w][g] - M);
+      L = fmaf(s_l[w][g], sc, L);
+      O = fmaf(s_o[w][g][d], sc, O);
+    }
+    const float val = (L > 0.f) ? O / L : 0.f;    // all pages of the chunk rejected: defined output
+    const size_t row_head = (size_t)r * p.Hq + head0 + g;
+    if (p.n_chunks == 1) {
+      p.out[row_head * D + d] = __bfloat16_as_ushort(__float2bfloat16_rn(val));
+      if (p.lse && d == 0) p.lse[row_head] = (M + log2f(L)) * 0.6931471805599453f;
+    } else {
+      p.part_o[(row_head * p.n_chunks + c) * D + d] = val;
+      if (d == 0) p.part_lse[row_head * p.n_chunks + c] = M + log2f(L);
+    }
+  }
+}
+
+// Merge the chunk partials of one (row, head): lse = log2 sum 2^lse_c,
+// o = sum 2^(lse_c - lse) o_c.  One warp per (row, head), lanes over head_dim.
+template <int D>
+__global__ void __launch_bounds__(128) decode_merge_kernel(const DecodeParams p) {
+  constexpr int EPL = D / 32;
+  const int lane = threadIdx.x & 31;
+  const size_t row_head = (size_t)blockIdx.x * 4 + (threadIdx.x >> 5);
+  if (row_head >= (size_t)p.R * p.Hq) return;
+  const int r = (int)(row_head / p.Hq);
+  const int len = __ldg(p.row_len + r);
+  uint16_t* out = p.out + row_head * D + lane * EPL;
+  if (len <= 0) {
+#pragma unroll
+    for (int e = 0; e < EPL; ++e) out[e] = 0;
+    if (p.lse && lane == 0) p.lse[row_head] = -INFINITY;
+    return;
+  }
+  const int nc = (len + p.chunk_tokens - 1) / p.chunk_tokens;
+  const float* pl = p.part_lse + row_head * p.n_chunks;
+  const float* po = p.part_o + row_head * p.n_chunks * D + lane * EPL;
+  float M = -INFINITY;
+  for (int c = 0; c < nc; ++c) M = fmaxf(M, pl[c]);
+  float L = 0.f, acc[EPL];
+#pragma unroll
+  for (int e = 0; e < EPL; ++e) acc[e] = 0.f;
+  for (int c = 0; c < nc; ++c) {
+    const float w = exp2f(pl[c] - M);
+    L += w;
+#pragma unroll
+    for (int e = 0; e < EPL; ++e) acc[e] = fmaf(w, po[(size_t)c * D + e], acc[e]);
+  }
+  const float inv = 1.f / L;
+#pragma unroll
+  for (int e = 0; e < EPL; ++e) out[e] = __bfloat16_as_ushort(__float2bfloat16_rn(acc[e] * inv));
+  if (p.lse && lane == 0) p.lse[row_head] = (M + log2f(L)) * 0.6931471805599453f;
+}
+
+DecodePlan plan_decode(int rows, int Hq, int Hkv, int D, int max_len) {
+  DecodePlan pl;
+  const int G = Hq / Hkv;
+  pl.group_tile = G >= 4 ? 4 : G;
+  if (G % 4 != 0 && G > 4) pl.group_tile = (G % 3 == 0) ? 3 : 4;
+  pl.gsplit = (G + pl.group_tile - 1) / pl.group_tile;
+  if (max_len < 1) max_len = 1;
+  // aim for ~32 CTAs per SM over the launch so ragged lengths even out, but keep a
+  // chunk between 256 and 2048 tokens (128 KB .. 1 MB of K+V at head_dim 128)
+  const long long ctas_per_chunkless = (long long)rows * Hkv * pl.gsplit;
+  long long want_chunks = (148LL * 32 + ctas_per_chunkless - 1) / ctas_per_chunkless;
+  if (want_chunks < 1) want_chunks = 1;
+  long long chunk = (max_len + want_chunks - 1) / want_chunks;
+  if (chunk < 256) chunk = 256;
+  if (chunk > 2048) chunk = 2048;
+  chunk = (chunk + 63) / 64 * 64;
+  pl.chunk_tokens = (int)chunk;
+  pl.n_chunks = (max_len + pl.chunk_tokens - 1) / pl.chunk_tokens;
+  pl.part_o_bytes = pl.n_chunks > 1 ? (size_t)rows * Hq * pl.n_chunks * D * sizeof(float) : 0;
+  pl.part_lse_bytes = pl.n_chunks > 1 ? ((size_t)rows * Hq * pl.n_chunks * sizeof(float) + 255) / 256 * 256 : 0;
+  return pl;
+}
+
+template <int D>
+static efim_status launch_decode_d(const DecodeParams& p, const DecodePlan& pl, cudaStream_t s) {
+  dim3 grid(p.R, p.Hkv * pl.gsplit, pl.n_chunks);
+  switch (pl.group_tile) {
+    case 1: decode_splitkv_kernel<D, 1><<<grid, 128, 0, s>>>(p); break;
+    case 2: decode_splitkv_kernel<D, 2><<<grid, 128, 0, s>>>(p); break;
+    case 3: decode_splitkv_kernel<D, 3><<<grid, 128, 0, s>>>(p); break;
+    default: decode_splitkv_kernel<D, 4><<<grid, 128, 0, s>>>(p); break;
+  }
+  EFIM_CUDA_TRY(cudaGetLastError());
+  if (pl.n_chunks > 1) {
+    const unsigned blocks = (unsigned)(((size_t)p.R * p.Hq + 3) / 4);
+    decode_merge_kernel<D><<<blocks, 128, 0, s>>>(p);
+    EFIM_CUDA_TRY(cudaGetLastError());
+  }
+  return EFIM_OK;
+}
+
+efim_status launch_decode(const DecodeParams& p, const DecodePlan& pl, int D, cudaStream_t s) {
+  if (p.R == 0) return EFIM_OK;
+  if (p.R > 2147483647 / 4 || p.Hkv * pl.gsplit > 65535 || pl.n_chunks > 65535) return EFIM_ERR_UNSUPPORTED;
+  return D == 128 ? launch_decode_d<128>(p, pl, s) : launch_decode_d<64>(p, pl, s);
+}
+
+}  // namespace efim
+
+extern "C" size_t efim_decode_workspace_bytes(const efim_cache_desc* cache, int32_t batch, int32_t max_ctx_len) {
+  if (efim::check_cache(cache) != EFIM_OK || batch <= 0) return 0;
+  const efim::DecodePlan pl = efim::plan_decode(batch, cache->num_q_heads, cache->num_kv_heads, cache->head_dim,
+                                                max_ctx_len);
+  return pl.part_o_bytes + pl.part_lse_bytes;
+}
+
+extern "C" efim_status efim_decode_attn(const efim_cache_desc* cache, int32_t batch, const int32_t* d_ctx_len,
+                                        int32_t max_ctx_len, const int32_t* d_block_table,
+                                        int32_t max_pages_per_seq, const void* d_q, void* d_out, float* d_lse,
+                                        float sm_scale, void* d_workspace, size_t workspace_bytes,
+                                        int32_t* d_status, void* stream) {
+  efim_status st = efim::check_cache(cache);
+  if (st != EFIM_OK) return st;
+  if (batch < 0 || max_pages_per_seq <= 0) return EFIM_ERR_INVALID_ARG;
+  if (batch == 0) return EFIM_OK;
+  if (!d_ctx_len || !d_block_table || !d_q || !d_out) return EFIM_ERR_INVALID_ARG;
+  if ((reinterpret_cast<uintptr_t>(d_q) | reinterpret_cast<uintptr_t>(d_out)) & 15) return EFIM_ERR_INVALID_ARG;
+  const long long cap = (long long)max_pages_per_seq * cache->page_size;
+  if (max_ctx_len <= 0) max_ctx_len = (int32_t)(cap > 2147483647LL ? 2147483647LL : cap);
+  if (max_ctx_len > cap) return EFIM_ERR_OUT_OF_RANGE;
+  const efim::DecodePlan pl = efim::plan_decode(batch, cache->num_q_heads, cache->num_kv_heads, cache->head_dim,
+                                                max_ctx_len);
+  const size_t need = pl.part_o_bytes + pl.part_lse_bytes;
+  if (need > 0) {
+    if (!d_workspace || workspace_bytes < need) return EFIM_ERR_WORKSPACE;
+    if (reinterpret_cast<uintptr_t>(d_workspace) & 255) return EFIM_ERR_INVALID_ARG;
+  }
+  efim::DecodeParams p{};
+  p.q = static_cast<const uint16_t*>(d_q);
+  p.k_pool = static_cast<const uint16_t*>(cache->d_k_pool);
+  p.v_pool = static_cast<const uint16_t*>(cache->d_v_pool);
+  p.row_len = d_ctx_len;
+  p.row_seq = nullptr;
+  p.block_table = d_block_table;
+  p.out = static_cast<uint16_t*>(d_out);
+  p.lse = d_lse;
+  p.part_lse = static_cast<float*>(d_workspace);
+  p.part_o = need ? reinterpret_cast<float*>(static_cast<char*>(d_workspace) + pl.part_lse_bytes) : nullptr;
+  p.status = d_status;
+  p.R = batch;
+  p.Hq = cache->num_q_heads;
+  p.Hkv = cache->num_kv_heads;
+  p.max_pages_per_seq = max_pages_per_seq;
+  p.num_pages = cache->num_pages;
+  p.chunk_tokens = pl.chunk_tokens;
+  p.n_chunks = pl.n_chunks;
+  const float scale = sm_scale > 0.f ? sm_scale : 1.0f / sqrtf((float)cache->head_dim);
+  p.scale_log2 = scale * 1.4426950408889634f;
+  return efim::launch_decode(p, pl, cache->head_dim, static_cast<cudaStream_t>(stream));
+}

@@ -1,0 +1,35 @@
+// Internal interface of the split-KV row-attention kernels (shared by the
+// decode entry point and the small-row path of append-prefill).
+#pragma once
+#include "common.cuh"
+
+namespace efim {
+
+struct DecodeParams {
+  const uint16_t* q;          // [R][Hq][D] bf16
+  const uint16_t* k_pool;     // [pages][Hkv][16][D]
+  const uint16_t* v_pool;
+  const int32_t* row_len;     // [R] keys visible to row r: [0, row_len[r])
+  const int32_t* row_seq;     // [R] block-table row of r, or null for identity
+  const int32_t* block_table; // [*][max_pages_per_seq]
+  uint16_t* out;              // [R][Hq][D] bf16
+  float* lse;                 // [R][Hq] natural log, or null
+  float* part_o;              // [R][Hq][n_chunks][D]   (n_chunks > 1)
+  float* part_lse;            // [R][Hq][n_chunks]      base-2 log
+  int32_t* status;
+  int R, Hq, Hkv, max_pages_per_seq, num_pages, chunk_tokens, n_chunks;
+  float scale_log2;           // sm_scale * log2(e)
+};
+
+struct DecodePlan {
+  int group_tile;             // q heads of one kv head handled per CTA (<= 4)
+  int gsplit;                 // CTAs per kv head
+  int chunk_tokens;           // keys per chunk (multiple of 64)
+  int n_chunks;
+  size_t part_o_bytes, part_lse_bytes;
+};
+
+DecodePlan plan_decode(int rows, int Hq, int Hkv, int D, int max_len);
+efim_status launch_decode(const DecodeParams& p, const DecodePlan& pl, int D, cudaStream_t s);
+
+}  // namespace efim

@@ -1,0 +1,207 @@
+// efim_kv_append: rotary embedding of the new tokens' q/k fused with the scatter
+// of k/v into the paged cache (EFIM Sec. 1: only the `inc` tokens are new and
+// they follow `<P>prefix<S>suffix<M>`, so token i of sequence s has position
+// cached_len[s] + i).  Pure streaming: every byte is read once and written once.
+#include "common.cuh"
+#include <math.h>
+
+namespace efim {
+
+struct KvAppendParams {
+  uint16_t* q;              // [T][Hq][D] in/out, may be null
+  const uint16_t* k_new;    // [T][Hkv][D]
+  const uint16_t* v_new;
+  uint16_t* k_pool;         // [pages][Hkv][P][D]
+  uint16_t* v_pool;
+  const int32_t* cached_len;
+  const int32_t* q_indptr;
+  const int32_t* block_table;
+  const float* cos_sin;     // [max_position][D] or null
+  int32_t* status;
+  int batch, max_pages_per_seq, total_new_tokens;
+  int num_pages, Hq, Hkv, max_position, interleaved;
+};
+
+// Rotate 8 (a, b) pairs held in two 16-byte vectors: a' = a c - b s, b' = b c + a s.
+__device__ __forceinline__ void rotate8(uint4& va, uint4& vb, const float* c, const float* s) {
+  uint32_t* a = reinterpret_cast<uint32_t*>(&va);
+  uint32_t* b = reinterpret_cast<uint32_t*>(&vb);
+#pragma unroll
+  for (int i = 0; i < 4; ++i) {
+    float a0 = bf16lo(a[i]), a1 = bf16hi(a[i]);
+    float b0 = bf16lo(b[i]), b1 = bf16hi(b[i]);
+    float ra0 = fmaf(a0, c[2 * i], -(b0 * s[2 * i]));
+    float ra1 = fmaf(a1, c[2 * i + 1], -(b1 * s[2 * i + 1]));
+    float rb0 = fmaf(b0, c[2 * i], a0 * s[2 * i]);
+    float rb1 = fmaf(b1, c[2 * i + 1], a1 * s[2 * i + 1]);
+    a[i] = pack_bf16x2(ra0, ra1);
+    b[i] = pack_bf16x2(rb0, rb1);
+  }
+}
+
+// Interleaved pairing: one 16-byte vector holds 4 pairs (2f, 2f+1).
+__device__ __forceinline__ void rotate4_interleaved(uint4& v, const float* c, const float* s) {
+  uint32_t* w = reinterpret_cast<uint32_t*>(&v);
+#pragma unroll
+  for (int i = 0; i < 4; ++i) {
+    float a = bf16lo(w[i]), b = bf16hi(w[i]);
+    float ra = fmaf(a, c[i], -(b * s[i]));
+    float rb = fmaf(b, c[i], a * s[i]);
+    w[i] = pack_bf16x2(ra, rb);
+  }
+}
+
+// One CTA per new token.  Work units of the token:
+//   rotate-half: (head, j) with j < D/16 -> vectors j and j + D/16 of that head (q heads then k heads)
+//   interleaved: (head, j) with j < D/8
+//   v copy:      (kv head, j) with j < D/8
+template <int D>
+__global__ void __launch_bounds__(256) kv_append_kernel(const KvAppendParams p) {
+  constexpr int VEC = D / 8;            // 16-byte vectors per head row
+  constexpr int HALF = VEC / 2;
+  const int t = blockIdx.x;
+  // sequence of this token: last s with q_indptr[s] <= t
+  int lo = 0, hi = p.batch;
+  while (hi - lo > 1) {
+    int mid = (lo + hi) >> 1;
+    if (__ldg(p.q_indptr + mid) <= t) lo = mid; else hi = mid;
+  }
+  const int s = lo;
+  const int pos = __ldg(p.cached_len + s) + (t - __ldg(p.q_indptr + s));
+  const int page_idx = pos >> 4;
+  int err = 0;
+  int page = -1;
+  if (pos < 0 || page_idx >= p.max_pages_per_seq || (p.cos_sin && pos >= p.max_position)) {
+    err = EFIM_DEV_BAD_POSITION;
+  } else {
+    page = __ldg(p.block_table + (size_t)s * p.max_pages_per_seq + page_idx);
+    if (page < 0 || page >= p.num_pages) err = EFIM_DEV_BAD_PAGE;
+  }
+  if (err) {
+    if (threadIdx.x == 0 && p.status) atomicOr(p.status, err);
+    return;
+  }
+  const int slot = pos & 15;
+  const size_t pool_tok = ((size_t)page * p.Hkv) * 16 * D + (size_t)slot * D;   // + h * 16 * D
+  const uint4* kin = reinterpret_cast<const uint4*>(p.k_new + (size_t)t * p.Hkv * D);
+  const uint4* vin = reinterpret_cast<const uint4*>(p.v_new + (size_t)t * p.Hkv * D);
+  uint4* qio = p.q ? reinterpret_cast<uint4*>(p.q + (size_t)t * p.Hq * D) : nullptr;
+  const int nq = p.q ? p.Hq : 0;
+
+  // v: straight copy into the page slot
+  for (int u = threadIdx.x; u < p.Hkv * VEC; u += blockDim.x) {
+    const int h = u / VEC, j = u % VEC;
+    uint4 v = ldg_stream(vin + u);
+    *reinterpret_cast<uint4*>(p.v_pool + pool_tok + (size_t)h * 16 * D + j * 8) = v;
+  }
+  if (!p.cos_sin) {
+    for (int u = threadIdx.x; u < p.Hkv * VEC; u += blockDim.x) {
+      const int h = u / VEC, j = u % VEC;
+      uint4 v = ldg_stream(kin + u);
+      *reinterpret_cast<uint4*>(p.k_pool + pool_tok + (size_t)h * 16 * D + j * 8) = v;
+    }
+    return;
+  }
+  const float* cs = p.cos_sin + (size_t)pos * D;     // cos[0..D/2) then sin[0..D/2)
+  if (!p.interleaved) {
+    const int units = (nq + p.Hkv) * HALF;
+    for (int u = threadIdx.x; u < units; u += blockDim.x) {
+      const int h = u / HALF, j = u % HALF;
+      float c[8], sn[8];
+      *reinterpret_cast<float4*>(c) = __ldg(reinterpret_cast<const float4*>(cs + j * 8));
+      *reinterpret_cast<float4*>(c + 4) = __ldg(reinterpret_cast<const float4*>(cs + j * 8 + 4));
+      *reinterpret_cast<float4*>(sn) = __ldg(reinterpret_cast<const float4*>(cs + D / 2 + j * 8));
+      *reinterpret_cast<float4*>(sn + 4) = __ldg(reinterpret_cast<const float4*>(cs + D / 2 + j * 8 + 4));
+      if (h < nq) {
+        uint4 a = qio[h * VEC + j], b = qio[h * VEC + j + HALF];
+        rotate8(a, b, c, sn);
+        qio[h * VEC + j] = a;
+        qio[h * VEC + j + HALF] = b;
+      } else {
+        const int hk = h - nq;
+        uint4 a = ldg_stream(kin + hk * VEC + j), b = ldg_stream(kin + hk * VEC + j + HALF);
+        rotate8(a, b, c, sn);
+        uint16_t* dst = p.k_pool + pool_tok + (size_t)hk * 16 * D;
+        *reinterpret_cast<uint4*>(dst + j * 8) = a;
+        *reinterpret_cast<uint4*>(dst + (j + HALF) * 8) = b;
+      }
+    }
+  } else {
+    const int units = (nq + p.Hkv) * VEC;
+    for (int u = threadIdx.x; u < units; u += blockDim.x) {
+      const int h = u / VEC, j = u % VEC;
+      float c[4], sn[4];
+      *reinterpret_cast<float4*>(c) = __ldg(reinterpret_cast<const float4*>(cs + j * 4));
+      *reinterpret_cast<float4*>(sn) = __ldg(reinterpret_cast<const float4*>(cs + D / 2 + j * 4));
+      if (h < nq) {
+        uint4 a = qio[h * VEC + j];
+        rotate4_interleaved(a, c, sn);
+        qio[h * VEC + j] = a;
+      } else {
+        const int hk = h - nq;
+        uint4 a = ldg_stream(kin + hk * VEC + j);
+        rotate4_interleaved(a, c, sn);
+        *reinterpret_cast<uint4*>(p.k_pool + pool_tok + (size_t)hk * 16 * D + j * 8) = a;
+      }
+    }
+  }
+}
+
+}  // namespace efim
+
+extern "C" efim_status efim_rope_table_build(double base, int32_t head_dim, int32_t max_position, float* h_out) {
+  if (!h_out || head_dim <= 0 || (head_dim & 1) || max_position <= 0 || !(base > 0.0)) return EFIM_ERR_INVALID_ARG;
+  const int half = head_dim / 2;
+  for (int f = 0; f < half; ++f) {
+    const double theta = pow(base, -2.0 * (double)f / (double)head_dim);
+    for (int p = 0; p < max_position; ++p) {
+      const double ang = (double)p * theta;
+      h_out[(size_t)p * head_dim + f] = (float)cos(ang);
+      h_out[(size_t)p * head_dim + half + f] = (float)sin(ang);
+    }
+  }
+  return EFIM_OK;
+}
+
+extern "C" efim_status efim_kv_append(const efim_cache_desc* cache, const efim_batch_desc* batch,
+                                      const efim_rope_desc* rope, void* d_q, const void* d_k_new,
+                                      const void* d_v_new, int32_t* d_status, void* stream) {
+  efim_status st = efim::check_cache(cache);
+  if (st != EFIM_OK) return st;
+  st = efim::check_batch(cache, batch, false);
+  if (st != EFIM_OK) return st;
+  if (batch->batch == 0 || batch->total_new_tokens == 0) return EFIM_OK;
+  if (!d_k_new || !d_v_new) return EFIM_ERR_INVALID_ARG;
+  if ((reinterpret_cast<uintptr_t>(d_k_new) | reinterpret_cast<uintptr_t>(d_v_new) |
+       reinterpret_cast<uintptr_t>(d_q)) & 15) return EFIM_ERR_INVALID_ARG;
+  efim::KvAppendParams p{};
+  p.q = static_cast<uint16_t*>(d_q);
+  p.k_new = static_cast<const uint16_t*>(d_k_new);
+  p.v_new = static_cast<const uint16_t*>(d_v_new);
+  p.k_pool = static_cast<uint16_t*>(cache->d_k_pool);
+  p.v_pool = static_cast<uint16_t*>(cache->d_v_pool);
+  p.cached_len = batch->d_cached_len;
+  p.q_indptr = batch->d_q_indptr;
+  p.block_table = batch->d_block_table;
+  p.cos_sin = nullptr;
+  if (rope && rope->d_cos_sin) {
+    if (rope->max_position <= 0 || (reinterpret_cast<uintptr_t>(rope->d_cos_sin) & 15)) return EFIM_ERR_INVALID_ARG;
+    p.cos_sin = rope->d_cos_sin;
+    p.max_position = rope->max_position;
+    p.interleaved = rope->interleaved;
+  }
+  p.status = d_status;
+  p.batch = batch->batch;
+  p.max_pages_per_seq = batch->max_pages_per_seq;
+  p.total_new_tokens = batch->total_new_tokens;
+  p.num_pages = cache->num_pages;
+  p.Hq = cache->num_q_heads;
+  p.Hkv = cache->num_kv_heads;
+  cudaStream_t s = static_cast<cudaStream_t>(stream);
+  if (cache->head_dim == 128)
+    efim::kv_append_kernel<128><<<batch->total_new_tokens, 256, 0, s>>>(p);
+  else
+    efim::kv_append_kernel<64><<<batch->total_new_tokens, 256, 0, s>>>(p);
+  EFIM_CUDA_TRY(cudaGetLastError());
+  return EFIM_OK;
+}

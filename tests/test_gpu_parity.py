@@ -1,0 +1,211 @@
+"""GPU parity: the CUDA library (through the C ABI) against the CPU oracle on the
+same seeded inputs.  Scatter/layout bit-exact; RoPE within one bf16 ulp; attention
+outputs max abs <= 2e-2 and mean abs <= 2e-3 (bf16 operands, fp32 accumulation)."""
+import numpy as np
+import pytest
+import torch
+
+from efim_synth import make_workload
+from oracle import efim_oracle as orc
+
+pytestmark = pytest.mark.gpu
+
+
+def _harness():
+    import tests.gpu_harness as H
+    return H
+
+
+def _check_turn(w, seqs=None, interleaved=False, use_rope=True, sm_scale=None):
+    H = _harness()
+    dw = H.DeviceWorkload(w, interleaved=interleaved, use_rope=use_rope)
+    dw.gpu_kv_append()
+    dw.gpu_prefill(0.0 if sm_scale is None else sm_scale)
+    torch.cuda.synchronize()
+    assert int(dw.status.item()) == 0
+    ref = dw.oracle_turn(seqs, sm_scale)
+    # --- cache contents of every page these sequences own
+    for r, s in enumerate(ref["seqs"]):
+        pg = w.pages_of(s)
+        want_k = ref["k_pool"][ref["bt"][r, :len(pg)]]
+        want_v = ref["v_pool"][ref["bt"][r, :len(pg)]]
+        got_k = dw.pages_from_device("k", pg)
+        got_v = dw.pages_from_device("v", pg)
+        assert np.array_equal(got_v, want_v), "V pages must match bit for bit"
+        if use_rope:
+            H.assert_rope_close(got_k, want_k, "K pages")
+            # slots not written this turn are untouched: exact
+            C, N = int(w.cached_len[s]), int(w.new_len[s])
+            tok = np.arange(len(pg) * w.page_size)
+            old = (tok < C) | (tok >= C + N)
+            gk = np.transpose(got_k, (0, 2, 1, 3)).reshape(len(tok), -1)
+            wk = np.transpose(want_k, (0, 2, 1, 3)).reshape(len(tok), -1)
+            assert np.array_equal(gk[old], wk[old])
+        else:
+            assert np.array_equal(got_k, want_k)
+    # --- rotated q
+    got_q = H.torch_to_bits(dw.q)[ref["rows"]]
+    if use_rope:
+        H.assert_rope_close(got_q, ref["q_rot"], "rotated q")
+    else:
+        assert np.array_equal(got_q, ref["q_rot"])
+    # --- attention
+    got_o = H.torch_to_bits(dw.out)[ref["rows"]]
+    H.assert_attn_close(got_o, ref["o"], f"{w.name} append-prefill")
+    got_lse = dw.lse.cpu().numpy()[ref["rows"]]
+    assert np.abs(got_lse - ref["lse"]).max(initial=0) <= H.LSE_TOL
+    return dw, ref
+
+
+def test_cfg1_turn_and_decode_steps():
+    H = _harness()
+    import paper_2505_21889_b200 as efim
+    w = make_workload("cfg1")
+    dw, ref = _check_turn(w)
+    # 8 decode steps: append one token, attend over everything so far
+    kp, vp, bt = ref["k_pool"], ref["v_pool"], ref["bt"]
+    ctx = (w.cached_len + w.new_len).astype(np.int32)
+    B = w.batch
+    d_bt = dw.batch.d_block_table
+    for step in range(w.decode_steps):
+        q, k, v = w.decode_qkv(step)
+        one = np.ones(B, np.int32)
+        q_rot = orc.kv_append(kp, vp, bt, ctx, one, q, k, v, w.rope_base)
+        ctx = ctx + 1
+        o, lse = orc.decode_attention(q_rot, kp, vp, bt, ctx, w.num_q_heads)
+        sb = efim.Batch(ctx - 1, one, d_bt)
+        dq, dk, dv = H.bits_to_torch(q), H.bits_to_torch(k), H.bits_to_torch(v)
+        efim.efim_kv_append(dw.cache, sb, dw.rope, dq, dk, dv, dw.status)
+        d_ctx = torch.from_numpy(ctx).cuda()
+        out = torch.empty_like(dq)
+        lse_d = torch.empty((B, w.num_q_heads), dtype=torch.float32, device="cuda")
+        nbytes = efim.efim_decode_workspace_bytes(dw.cache, B, int(ctx.max()))
+        ws = torch.empty(max(nbytes, 256), dtype=torch.uint8, device="cuda")
+        efim.efim_decode_attn(dw.cache, B, d_ctx, int(ctx.max()), d_bt, dq, out, lse_d, 0.0, ws, dw.status)
+        torch.cuda.synchronize()
+        assert int(dw.status.item()) == 0
+        H.assert_rope_close(H.torch_to_bits(dq), q_rot, "decode q")
+        H.assert_attn_close(H.torch_to_bits(out), o, f"cfg1 decode step {step}")
+        assert np.abs(lse_d.cpu().numpy() - lse).max() <= H.LSE_TOL
+    pg = w.pages_of(0)
+    assert np.array_equal(dw.pages_from_device("v", pg), vp[bt[0, :len(pg)]])
+
+
+@pytest.mark.parametrize("name", ["cfg2", "cfg3", "cfg4a", "cfg4b", "cfg4b_3072"])
+def test_small_configs_all_rows(name):
+    _check_turn(make_workload(name, small=True))
+
+
+@pytest.mark.parametrize("interleaved,use_rope", [(True, True), (False, False)])
+def test_cfg1_rope_variants(interleaved, use_rope):
+    _check_turn(make_workload("cfg1"), interleaved=interleaved, use_rope=use_rope)
+
+
+def test_custom_scale():
+    _check_turn(make_workload("cfg1"), sm_scale=0.2)
+
+
+def _custom(Hq, Hkv, D, cached, new, seed=7, extra=3):
+    from efim_synth.workloads import Workload, _block_table
+    cached = np.asarray(cached, np.int32)
+    new = np.asarray(new, np.int32)
+    rng = np.random.default_rng([seed, 99])
+    pages = int((-(-(cached + new + extra) // 16)).sum()) + 7
+    bt = _block_table(rng, pages, cached + new + extra, 16)
+    return Workload(f"custom{Hq}_{Hkv}_{D}", seed, Hq, Hkv, D, 16, pages, 10000.0, cached, new, bt, decode_steps=extra)
+
+
+@pytest.mark.parametrize("Hq,Hkv,D,cached,new", [
+    (4, 4, 64, [237], [16]),                 # cached length not page aligned
+    (8, 2, 128, [0, 5, 300], [33, 1, 130]),  # nothing cached; one new token; spans tiles
+    (7, 1, 128, [100, 17], [40, 3]),         # group of 7
+    (14, 2, 64, [64, 0], [0, 50]),           # a sequence with no new tokens
+    (6, 2, 128, [15, 16, 17], [17, 16, 15]), # around page edges
+    (1, 1, 64, [1], [1]),
+    (16, 1, 128, [50], [9]),                 # group of 16
+])
+def test_edge_shapes(Hq, Hkv, D, cached, new):
+    _check_turn(_custom(Hq, Hkv, D, cached, new))
+
+
+@pytest.mark.parametrize("name", ["cfg5"])
+def test_decode_loop_small(name):
+    H = _harness()
+    import paper_2505_21889_b200 as efim
+    w = make_workload(name, small=True)
+    dw = H.DeviceWorkload(w)
+    kp, vp, bt, seqs = w.compact_host_pool()
+    ctx = w.cached_len.astype(np.int32).copy()
+    B = w.batch
+    d_bt = dw.batch.d_block_table
+    max_ctx = int(ctx.max()) + w.decode_steps
+    nbytes = efim.efim_decode_workspace_bytes(dw.cache, B, max_ctx)
+    ws = torch.empty(max(nbytes, 256), dtype=torch.uint8, device="cuda")
+    one = np.ones(B, np.int32)
+    for step in range(w.decode_steps):
+        q, k, v = w.decode_qkv(step)
+        q_rot = orc.kv_append(kp, vp, bt, ctx, one, q, k, v, w.rope_base)
+        sb = efim.Batch(ctx, one, d_bt)
+        ctx = ctx + 1
+        o, lse = orc.decode_attention(q_rot, kp, vp, bt, ctx, w.num_q_heads)
+        dq, dk, dv = H.bits_to_torch(q), H.bits_to_torch(k), H.bits_to_torch(v)
+        efim.efim_kv_append(dw.cache, sb, dw.rope, dq, dk, dv, dw.status)
+        d_ctx = torch.from_numpy(ctx).cuda()
+        out = torch.empty_like(dq)
+        lse_d = torch.empty((B, w.num_q_heads), dtype=torch.float32, device="cuda")
+        efim.efim_decode_attn(dw.cache, B, d_ctx, max_ctx, d_bt, dq, out, lse_d, 0.0, ws, dw.status)
+        torch.cuda.synchronize()
+        assert int(dw.status.item()) == 0
+        H.assert_attn_close(H.torch_to_bits(out), o, f"{name} decode step {step}")
+        assert np.abs(lse_d.cpu().numpy() - lse).max() <= H.LSE_TOL
+
+
+def test_decode_zero_length_and_bad_page_flag():
+    H = _harness()
+    import paper_2505_21889_b200 as efim
+    w = _custom(4, 2, 128, [40, 0, 90], [0, 0, 0])
+    dw = H.DeviceWorkload(w)
+    ctx = torch.tensor([40, 0, 90], dtype=torch.int32, device="cuda")
+    q = H.bits_to_torch(w._normal_bits(5, (3, 4, 128)))
+    out = torch.full_like(q, 7.0)
+    lse = torch.zeros((3, 4), dtype=torch.float32, device="cuda")
+    ws = torch.empty(max(efim.efim_decode_workspace_bytes(dw.cache, 3, 96), 256), dtype=torch.uint8, device="cuda")
+    efim.efim_decode_attn(dw.cache, 3, ctx, 96, dw.batch.d_block_table, q, out, lse, 0.0, ws, dw.status)
+    torch.cuda.synchronize()
+    assert int(dw.status.item()) == 0
+    assert torch.all(out[1] == 0) and torch.all(torch.isinf(lse[1])) and torch.all(lse[1] < 0)
+    # a block-table id outside the pool is reported, not dereferenced
+    bad = dw.batch.d_block_table.clone()
+    bad[2, 1] = w.num_pages + 5
+    efim.efim_decode_attn(dw.cache, 3, ctx, 96, bad, q, out, lse, 0.0, ws, dw.status)
+    torch.cuda.synchronize()
+    assert int(dw.status.item()) & 0x1
+    assert torch.isfinite(out.float()).all()
+
+
+def test_pages_outside_the_batch_are_untouched():
+    H = _harness()
+    w = make_workload("cfg2", small=True)
+    dw = H.DeviceWorkload(w)
+    used = set(w.block_table[w.block_table >= 0].tolist())
+    free = np.array([p for p in range(w.num_pages) if p not in used][:200])
+    before_k, before_v = dw.pages_from_device("k", free), dw.pages_from_device("v", free)
+    assert np.array_equal(before_k, w.page_bits("k", free))      # device fill == host fill
+    dw.gpu_kv_append()
+    dw.gpu_prefill()
+    torch.cuda.synchronize()
+    assert np.array_equal(dw.pages_from_device("k", free), before_k)
+    assert np.array_equal(dw.pages_from_device("v", free), before_v)
+
+
+def test_run_to_run_bit_reproducible():
+    H = _harness()
+    w = make_workload("cfg3", small=True)
+    outs = []
+    for _ in range(2):
+        dw = H.DeviceWorkload(w)
+        dw.gpu_kv_append()
+        dw.gpu_prefill()
+        torch.cuda.synchronize()
+        outs.append((H.torch_to_bits(dw.out), dw.lse.cpu().numpy()))
+    assert np.array_equal(outs[0][0], outs[1][0]) and np.array_equal(outs[0][1], outs[1][1])
