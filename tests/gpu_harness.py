@@ -30,10 +30,15 @@ def ordered(bits: np.ndarray) -> np.ndarray:
 
 
 def assert_rope_close(got_bits, want_bits, what):
-    """fp32 table + fp32 FMA against fp64-then-round: a result within ~2^-22 of a
-    rounding tie may land on the neighbouring bf16 value, never further."""
+    """fp32 table + fp32 FMA against fp64-then-round.  The fp32 result carries an
+    absolute error of a few 2^-24 * |input| (inputs are |x| < 8), so it either rounds
+    to the same bf16 value, to a neighbour when the exact result sits within that
+    error of a rounding tie, or - where a*cos and b*sin cancel and the result is
+    tiny - differs by that absolute error although it spans several tiny ulps."""
     d = np.abs(ordered(got_bits) - ordered(want_bits))
-    assert d.max(initial=0) <= 1, f"{what}: off by more than one bf16 ulp"
+    abs_err = np.abs(bf16_bits_to_f32(got_bits).astype(np.float64) - bf16_bits_to_f32(want_bits).astype(np.float64))
+    bad = (d > 1) & (abs_err > 4e-6)
+    assert not bad.any(), f"{what}: {int(bad.sum())} elements beyond one bf16 ulp and beyond fp32 rounding error"
     if d.size:
         assert (d == 0).mean() >= 0.99, f"{what}: only {(d == 0).mean():.4f} identical"
 
