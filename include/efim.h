@@ -15,8 +15,8 @@
  *
  * Conventions for every entry point
  *   - Pointers named d_* are DEVICE pointers, h_* are HOST pointers.  The caller
- *     owns all memory and the stream; the library allocates no device memory,
- *     keeps no state between calls and never synchronises the device.
+ *     owns all memory and the stream; the library allocates no device memory and,
+ *     apart from the fixed array of efim_decode_attn_static, keeps no state between calls; it never synchronises the device.
  *   - `stream` is a cudaStream_t passed as void* (NULL = default stream).  All
  *     work is enqueued on it; results are ready when the stream reaches that point.
  *   - bf16 tensors are raw 16-bit patterns.  Packed layouts, innermost last:
@@ -152,6 +152,35 @@ efim_status efim_decode_attn(const efim_cache_desc* cache, int32_t batch,
                              const void* d_q, void* d_out, float* d_lse, float sm_scale,
                              void* d_workspace, size_t workspace_bytes,
                              int32_t* d_status, void* stream);
+
+/*
+ * Allocation-free variant of efim_decode_attn (the paper has no counterpart; this is
+ * a convenience of this library).  For callers that cannot provide a workspace
+ * because they may not allocate device memory at all - a serving loop that has
+ * given every free byte to its KV pool, a plug-in handed only input and output
+ * pointers, a latency-critical thread that must not block in the allocator.  The
+ * chunk partials go to a fixed array of efim_decode_static_scratch_bytes() bytes
+ * (8 MiB) that lives inside the library on every GPU that loads it, from load to
+ * process exit.  Same arguments, results and errors as efim_decode_attn without the
+ * workspace pair, plus:
+ *   - EFIM_ERR_WORKSPACE if this (batch, heads, max_ctx_len) needs more than the
+ *     fixed array, i.e. efim_decode_workspace_bytes() > efim_decode_static_scratch_bytes();
+ *     use efim_decode_attn with your own workspace then.
+ *   - The first call on each device looks up the array's device address (no
+ *     allocation, but a runtime query): make that first call outside any stream
+ *     capture, with the device current.
+ *   - All calls on a device share the one array and it keeps the previous call's
+ *     partials.  Nothing has to be cleared (each call overwrites what it reads back),
+ *     but two calls whose kernels may overlap on the GPU - different streams without
+ *     an ordering between them - race on it.  Issue them on one stream or order them.
+ *   - Calls no cudaMalloc/cudaFree and no allocating library routine.
+ */
+size_t efim_decode_static_scratch_bytes(void);
+efim_status efim_decode_attn_static(const efim_cache_desc* cache, int32_t batch,
+                                    const int32_t* d_ctx_len, int32_t max_ctx_len,
+                                    const int32_t* d_block_table, int32_t max_pages_per_seq,
+                                    const void* d_q, void* d_out, float* d_lse, float sm_scale,
+                                    int32_t* d_status, void* stream);
 
 #ifdef __cplusplus
 }

@@ -7,5 +7,5 @@ from .binding import (  # noqa: F401
     EfimError, Cache, Batch, Rope, load_library, library_path, exported_symbols,
     efim_kv_append, efim_append_prefill_attn, efim_decode_attn,
     efim_prefill_workspace_bytes, efim_decode_workspace_bytes, efim_rope_table_build,
-    efim_strerror, efim_version,
+    efim_strerror, efim_version, efim_decode_attn_static, efim_decode_static_scratch_bytes,
 )

@@ -35,7 +35,8 @@ class _RopeDesc(Structure):
 
 EXPORTS = ("efim_strerror", "efim_version", "efim_rope_table_build", "efim_kv_append",
            "efim_prefill_workspace_bytes", "efim_append_prefill_attn",
-           "efim_decode_workspace_bytes", "efim_decode_attn")
+           "efim_decode_workspace_bytes", "efim_decode_attn",
+           "efim_decode_static_scratch_bytes", "efim_decode_attn_static")
 
 
 def library_path() -> str:
@@ -71,6 +72,11 @@ def load_library():
     lib.efim_decode_attn.argtypes = [POINTER(_CacheDesc), c_int32, c_void_p, c_int32, c_void_p, c_int32,
                                      c_void_p, c_void_p, c_void_p, c_float, c_void_p, c_size_t,
                                      c_void_p, c_void_p]
+    lib.efim_decode_static_scratch_bytes.restype = c_size_t
+    lib.efim_decode_static_scratch_bytes.argtypes = []
+    lib.efim_decode_attn_static.restype = ctypes.c_int
+    lib.efim_decode_attn_static.argtypes = [POINTER(_CacheDesc), c_int32, c_void_p, c_int32, c_void_p, c_int32,
+                                            c_void_p, c_void_p, c_void_p, c_float, c_void_p, c_void_p]
     _LIB = lib
     return lib
 
@@ -196,3 +202,19 @@ def efim_decode_attn(cache: Cache, batch: int, d_ctx_len, max_ctx_len, d_block_t
                                          _ptr(status), _stream_ptr(stream))
     if st != 0:
         raise EfimError(st, "efim_decode_attn")
+
+
+def efim_decode_static_scratch_bytes() -> int:
+    return int(load_library().efim_decode_static_scratch_bytes())
+
+
+def efim_decode_attn_static(cache: Cache, batch: int, d_ctx_len, max_ctx_len, d_block_table, q, out, lse=None,
+                            sm_scale=0.0, status=None, stream=None):
+    """efim_decode_attn for callers that cannot allocate a workspace: the chunk
+    partials use the library's fixed 8 MiB array (shared by all calls on the device)."""
+    st = load_library().efim_decode_attn_static(ctypes.byref(cache.desc), batch, _ptr(d_ctx_len), int(max_ctx_len),
+                                                _ptr(d_block_table), int(d_block_table.shape[1]), _ptr(q),
+                                                _ptr(out), _ptr(lse), float(sm_scale), _ptr(status),
+                                                _stream_ptr(stream))
+    if st != 0:
+        raise EfimError(st, "efim_decode_attn_static")
