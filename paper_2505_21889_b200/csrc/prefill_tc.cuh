@@ -1,0 +1,54 @@
+// Internal interface of the tensor-core append-prefill kernel.
+#pragma once
+#include <cuda.h>
+#include "common.cuh"
+
+namespace efim {
+namespace pf {
+
+constexpr int BM = 128;        // query rows per tile (one TMEM lane each)
+constexpr int BN = 128;        // keys per KV tile (8 pages)
+constexpr int NQ = 2;          // query tiles per CTA sharing one K/V stream
+constexpr int NSTAGE = 3;      // K/V ring entries
+constexpr int THREADS = 320;   // 8 softmax warps + TMA warp + MMA warp
+
+// One CTA's work: packed rows [row0, row0 + 256) of (seq, kv head) against KV tiles
+// [tile_begin, tile_end).  Packed row R = token * G + head-in-group.
+struct WorkItem {
+  int32_t seq, kvh, row0, tile_begin, tile_end;
+  int32_t chunk;               // >= 0: write a partial for this KV chunk; -1: final output
+  int32_t pad0, pad1;
+};
+
+struct Params {
+  const uint16_t* q;           // [T][Hq][D]
+  uint16_t* out;               // [T][Hq][D]
+  float* lse;                  // [T][Hq] or null
+  const int32_t* cached_len;
+  const int32_t* new_len;
+  const int32_t* q_indptr;
+  const int32_t* block_table;
+  const WorkItem* items;
+  const int32_t* split_tokens; // [batch] keys per KV chunk of a split sequence, 0 = not split
+  float* part_o;               // [T][Hq][s_max][D]
+  float* part_lse;             // [T][Hq][s_max]  base-2
+  int32_t* status;
+  int batch, total_new_tokens;
+  int Hq, Hkv, G, max_pages_per_seq, num_pages, s_max;
+  float scale_log2;
+};
+
+struct Plan {
+  int n_items;
+  int s_max;                   // largest KV split count (1 = no partials, no merge)
+  size_t items_bytes, split_bytes, part_lse_bytes, part_o_bytes;
+  size_t total() const { return items_bytes + split_bytes + part_lse_bytes + part_o_bytes; }
+};
+
+// Host: size the plan (items == nullptr) or fill `items`/`split_tokens` too.
+Plan make_plan(const efim_cache_desc* c, const efim_batch_desc* b, WorkItem* items, int32_t* split_tokens);
+
+efim_status launch(const efim_cache_desc* c, const Params& p, const Plan& pl, cudaStream_t s);
+
+}  // namespace pf
+}  // namespace efim
