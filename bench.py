@@ -79,7 +79,7 @@ class ClockSampler:
         try:
             self.proc = subprocess.Popen(
                 ["nvidia-smi", "-i", str(self.index), f"--query-gpu={self.FIELDS}",
-                 "--format=csv,noheader,nounits", "-lms", "100"],
+                 "--format=csv,noheader,nounits", "-lms", "20"],
                 stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
             self.thread = threading.Thread(target=self._pump, daemon=True)
             self.thread.start()
@@ -181,7 +181,7 @@ def run_reference(args):
     if rank != 0:
         return
     from efim_synth import make_workload
-    w = make_workload(args.workload)
+    w = make_workload(args.workload, batch=args.batch)
     q, k, v = w.new_qkv()
     dq, dk, dv = w.decode_qkv(0) if w.decode_steps > 0 else (None, None, None)
     seqs = pick_sample(w, 6e9)
@@ -232,7 +232,7 @@ def run_native(args):
     efim.load_library()                       # raises if the CUDA library is missing
 
     base_seed = {"cfg1": 0, "cfg2": 2, "cfg3": 3, "cfg4a": 4, "cfg4b": 4, "cfg4b_3072": 4, "cfg5": 5}[args.workload]
-    w = make_workload(args.workload, seed=base_seed + 1000 * rank if rank else None)
+    w = make_workload(args.workload, seed=base_seed + 1000 * rank if rank else None, batch=args.batch)
     cnt = workload_counts(w)
     B, Hq, Hkv, D = w.batch, w.num_q_heads, w.num_kv_heads, w.head_dim
     has_decode = w.decode_steps > 0
@@ -438,6 +438,7 @@ def main():
     ap.add_argument("--warmup", type=int, default=5)
     ap.add_argument("--impl", default="native", choices=["native", "reference"])
     ap.add_argument("--workload", default="cfg2")
+    ap.add_argument("--batch", type=int, default=None, help="override the sequence count of cfg2/cfg5")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     args = ap.parse_args()
     if args.impl == "reference":

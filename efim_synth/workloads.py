@@ -158,7 +158,9 @@ def _block_table(rng, num_pages, total_len, page_size):
     return bt
 
 
-def make_workload(name: str, small: bool = False, seed: Optional[int] = None) -> Workload:
+def make_workload(name: str, small: bool = False, seed: Optional[int] = None,
+                  batch: Optional[int] = None) -> Workload:
+    """`batch` overrides the number of sequences of cfg2/cfg5 (the pool shrinks or grows with it)."""
     if name not in WORKLOAD_NAMES:
         raise ValueError(f"unknown workload {name!r}; choose from {WORKLOAD_NAMES}")
     P = 16
@@ -181,9 +183,10 @@ def make_workload(name: str, small: bool = False, seed: Optional[int] = None) ->
             cached = _uniform_int(rng, 200, 800, 6)
             new = _uniform_int(rng, 32, 256, 6)
         else:
-            pages = 65536
-            cached = _uniform_int(rng, 2048, 8192, 16)
-            new = _uniform_int(rng, 32, 256, 16)
+            nb = 16 if batch is None else batch
+            pages = 65536 * nb // 16
+            cached = _uniform_int(rng, 2048, 8192, nb)
+            new = _uniform_int(rng, 32, 256, nb)
     elif name == "cfg3":
         sd = 3 if seed is None else seed
         Hq, Hkv, D, steps = 28, 4, 128, 0
@@ -234,7 +237,8 @@ def make_workload(name: str, small: bool = False, seed: Optional[int] = None) ->
             nb, pages, steps = 12, 4096, 4
             ctx = _uniform_int(rng, 300, 3000, nb)
         else:
-            nb, pages, steps = 256, 540672, 64
+            nb, steps = (256 if batch is None else batch), 64
+            pages = 2112 * nb
             ctx = _uniform_int(rng, 4096, 32768, nb)
         # the decode loop: step t appends one token at position ctx+t
         cached = ctx.astype(np.int32)
