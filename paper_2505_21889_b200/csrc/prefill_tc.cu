@@ -204,6 +204,14 @@ prefill_tc_kernel(const Params p, const __grid_constant__ CUtensorMap map_k, con
   const uint32_t tmem_S = tmem;                // S_t at columns [t*128, t*128+128)
   const uint32_t tmem_O = tmem + NQ * BN;      // O_t at columns [256 + t*D, ...)
 
+  // Register split: every warp of a warpgroup runs the same setmaxnreg; the service
+  // group releases first what the two softmax groups then take.
+  if (warp >= 8) {
+    asm volatile("setmaxnreg.dec.sync.aligned.u32 %0;" ::"n"(REGS_SERVICE));
+  } else {
+    asm volatile("setmaxnreg.inc.sync.aligned.u32 %0;" ::"n"(REGS_SOFTMAX));
+  }
+
   if (warp < 8) {
     // ============================================================ softmax groups
     const int t = warp >> 2;
@@ -248,9 +256,15 @@ prefill_tc_kernel(const Params p, const __grid_constant__ CUtensorMap map_k, con
           for (int c = 0; c < BN; ++c)
             if (kv0 + c >= vis) s[c] = 0xff800000u;         // -inf
         }
-        float mx = -INFINITY;
+        float mx8[8];
 #pragma unroll
-        for (int c = 0; c < BN; ++c) mx = fmaxf(mx, __uint_as_float(s[c]));
+        for (int a = 0; a < 8; ++a) mx8[a] = __uint_as_float(s[a]);
+#pragma unroll
+        for (int c = 8; c < BN; c += 8)
+#pragma unroll
+          for (int a = 0; a < 8; ++a) mx8[a] = fmaxf(mx8[a], __uint_as_float(s[c + a]));
+        const float mx = fmaxf(fmaxf(fmaxf(mx8[0], mx8[1]), fmaxf(mx8[2], mx8[3])),
+                               fmaxf(fmaxf(mx8[4], mx8[5]), fmaxf(mx8[6], mx8[7])));
         const float m_new = mx * p.scale_log2;
         // lazy rescale: keep the old reference maximum until it is off by more than 2^8
         const bool grow = m_new > m_ref + 8.f;
@@ -273,6 +287,7 @@ prefill_tc_kernel(const Params p, const __grid_constant__ CUtensorMap map_k, con
         }
         const float m_use = (m_ref == -INFINITY) ? 0.f : m_ref;
         const float neg_m = -m_use;
+        float ls[4] = {0.f, 0.f, 0.f, 0.f};
 #pragma unroll
         for (int c16 = 0; c16 < BN / 8; ++c16) {
           uint32_t w[4];
@@ -280,12 +295,13 @@ prefill_tc_kernel(const Params p, const __grid_constant__ CUtensorMap map_k, con
           for (int e = 0; e < 4; ++e) {
             const float p0 = ex2(fmaf(__uint_as_float(s[c16 * 8 + 2 * e]), p.scale_log2, neg_m));
             const float p1 = ex2(fmaf(__uint_as_float(s[c16 * 8 + 2 * e + 1]), p.scale_log2, neg_m));
-            l_sum += p0 + p1;
+            ls[e] += p0 + p1;
             w[e] = pack_bf16x2(p0, p1);
           }
           *reinterpret_cast<uint4*>(prow + (c16 >> 3) * L::HALF_BYTES + (((c16 & 7) ^ (r & 7)) << 4)) =
               make_uint4(w[0], w[1], w[2], w[3]);
         }
+        l_sum += (ls[0] + ls[1]) + (ls[2] + ls[3]);
         fence_async_smem();
         tc_fence_before();
         mbar_arrive(bar(BAR_P + t));
@@ -365,7 +381,7 @@ prefill_tc_kernel(const Params p, const __grid_constant__ CUtensorMap map_k, con
         for (int spin = 0; spin < (1 << 20) && !mbar_try(b, par); ++spin) {}
       }
     }
-  } else {
+  } else if (warp == 9) {
     // ============================================================ MMA issuer
     constexpr uint32_t IDESC_QK = instr_desc(BN, 0);
     constexpr uint32_t IDESC_PV = instr_desc(D, 1);
