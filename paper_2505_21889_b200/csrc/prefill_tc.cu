@@ -6,11 +6,11 @@
 // (sequence, kv head) as two 128-row tiles, and streams the visible K/V range in
 // tiles of 128 keys (8 pages):
 //   warp 8    TMA producer: walks the block table, one tiled bulk-tensor copy per
-//             (page, 64-dim half) into a 3-entry shared-memory ring (128B swizzle)
-//   warp 9    issues tcgen05.mma: S_t = Q_t K^T into TMEM, then O_t += P_t V
+//             (page, 64-dim half) into a 5-entry shared-memory ring (128B swizzle)
+//   warp 9    issues tcgen05.mma: S_t = Q_t K^T into TMEM, then O_t += P_t V (P from TMEM)
 //   warps 0-7 two softmax groups, one per query tile, one TMEM lane (row) per thread:
-//             S from TMEM, mask, running max with lazy rescale, exp2, P (bf16) to
-//             shared memory, final normalisation and store
+//             S from TMEM, mask, running max with lazy rescale, exp2, P (bf16) back to
+//             TMEM over S, final normalisation and store
 // Hand-offs are mbarriers; every wait is bounded and on expiry sets
 // EFIM_DEV_TIMEOUT and lets all roles run out their (fixed) loop counts.
 #include "prefill_tc.cuh"
@@ -79,6 +79,15 @@ __device__ __forceinline__ void umma_bf16(uint32_t d_tmem, uint64_t adesc, uint6
       "l"(adesc), "l"(bdesc), "r"(idesc), "r"(accumulate)
       : "memory");
 }
+// same with the A operand (P, bf16) read from tensor memory
+__device__ __forceinline__ void umma_bf16_ts(uint32_t d_tmem, uint32_t a_tmem, uint64_t bdesc, uint32_t idesc,
+                                             uint32_t accumulate) {
+  asm volatile(
+      "{\n.reg .pred p;\nsetp.ne.b32 p, %4, 0;\n"
+      "tcgen05.mma.cta_group::1.kind::f16 [%0], [%1], %2, %3, p;\n}\n" ::"r"(d_tmem),
+      "r"(a_tmem), "l"(bdesc), "r"(idesc), "r"(accumulate)
+      : "memory");
+}
 __device__ __forceinline__ void tma_load_4d(uint32_t dst, const CUtensorMap* map, uint32_t bar, int c0, int c1,
                                             int c2, int c3) {
   asm volatile(
@@ -139,17 +148,23 @@ struct Smem {
   static constexpr int HALVES = D / 64;
   static constexpr int HALF_BYTES = 128 * 128;                  // 16 KB
   static constexpr int Q_BYTES = HALVES * HALF_BYTES;
-  static constexpr int P_BYTES = 2 * HALF_BYTES;                // 128 keys = two 64-key halves
   static constexpr int KV_BYTES = HALVES * HALF_BYTES;
   static constexpr int Q_OFF = 0;
-  static constexpr int P_OFF = Q_OFF + NQ * Q_BYTES;
-  static constexpr int KV_OFF = P_OFF + NQ * P_BYTES;
+  static constexpr int KV_OFF = Q_OFF + NQ * Q_BYTES;
   static constexpr int BAR_OFF = KV_OFF + NSTAGE * KV_BYTES;
   static constexpr int TOTAL = BAR_OFF + 256 + 1024;            // + alignment slack
+  // epilogue exchange between the two softmax groups (re-uses the K/V ring)
+  static constexpr int XROW = D + 4;                            // floats per row, padded
+  static_assert(BM * XROW * 4 <= NSTAGE * KV_BYTES, "exchange buffer must fit in the ring");
 };
 // barrier slots (8 bytes each) inside the BAR_OFF block
 enum { BAR_Q = 0, BAR_S = 2, BAR_P = 4, BAR_O = 6, BAR_FULL = 8, BAR_EMPTY = 8 + NSTAGE, BAR_COUNT = 8 + 2 * NSTAGE };
 
+// Two softmax groups ("streams") run per CTA.  With more than 128 rows, stream t
+// owns query tile t and both walk every KV tile.  With 128 rows or fewer there is
+// one query tile; stream 0 takes the even KV tiles and stream 1 the odd ones, each
+// with its own running (max, sum, O), and the two states are merged at the end -
+// the tensor core then still works on one stream while the other does its softmax.
 template <int D>
 __global__ void __launch_bounds__(THREADS, 1)
 prefill_tc_kernel(const Params p, const __grid_constant__ CUtensorMap map_k, const __grid_constant__ CUtensorMap map_v) {
@@ -171,10 +186,12 @@ prefill_tc_kernel(const Params p, const __grid_constant__ CUtensorMap map_k, con
   const int tok0 = __ldg(p.q_indptr + it.seq);
   const int rows_total = N * G;
   const int rows_here = min(NQ * BM, rows_total - it.row0);
-  const int nq_active = rows_here > BM ? 2 : 1;
+  const bool dual = rows_here > BM;                          // two query tiles
   const int i_last = (it.row0 + rows_here - 1) / G;          // last token of this CTA
   const int kv_cap = C + i_last + 1;                         // keys any row here may see
   const int nt = it.tile_end - it.tile_begin;
+  const int cnt0 = dual ? nt : (nt + 1) >> 1;                // KV tiles of stream 0 / 1
+  const int cnt1 = dual ? nt : nt >> 1;
 
   if (tid == 0) {
     for (int t = 0; t < NQ; ++t) {
@@ -201,8 +218,8 @@ prefill_tc_kernel(const Params p, const __grid_constant__ CUtensorMap map_k, con
   __syncthreads();
   tc_fence_after();
   const uint32_t tmem = *tmem_slot;
-  const uint32_t tmem_S = tmem;                // S_t at columns [t*128, t*128+128)
-  const uint32_t tmem_O = tmem + NQ * BN;      // O_t at columns [256 + t*D, ...)
+  const uint32_t tmem_S = tmem;                // S of stream t at columns [t*128, t*128+128); P (bf16) re-uses its first 64
+  const uint32_t tmem_O = tmem + NQ * BN;      // O of stream t at columns [256 + t*D, ...)
 
   // Register split: every warp of a warpgroup runs the same setmaxnreg; the service
   // group releases first what the two softmax groups then take.
@@ -214,126 +231,163 @@ prefill_tc_kernel(const Params p, const __grid_constant__ CUtensorMap map_k, con
 
   if (warp < 8) {
     // ============================================================ softmax groups
-    const int t = warp >> 2;
-    if (t < nq_active) {
-      const int r = (warp & 3) * 32 + lane;                 // tile row == TMEM lane
-      const int R = it.row0 + t * BM + r;                   // packed row of the (seq, kv head)
-      const bool valid = R < rows_total;
-      const int i_tok = valid ? R / G : 0;
-      const int g = valid ? R - i_tok * G : 0;
-      const int vis = valid ? C + i_tok + 1 : 0;            // keys this row sees
-      const size_t row_off = ((size_t)(tok0 + i_tok) * p.Hq + (size_t)it.kvh * G + g) * D;
+    const int st = warp >> 2;                               // stream
+    const int my_cnt = st == 0 ? cnt0 : cnt1;
+    const int qt = dual ? st : 0;                           // query tile of this stream
+    const int r = (warp & 3) * 32 + lane;                   // tile row == TMEM lane
+    const int R = it.row0 + qt * BM + r;                    // packed row of the (seq, kv head)
+    const bool valid = R < rows_total;
+    const int i_tok = valid ? R / G : 0;
+    const int g = valid ? R - i_tok * G : 0;
+    const int vis = valid ? C + i_tok + 1 : 0;              // keys this row sees
+    const size_t row_off = ((size_t)(tok0 + i_tok) * p.Hq + (size_t)it.kvh * G + g) * D;
+    if (dual || st == 0) {
       // ---- Q row -> shared memory (swizzled), zero for rows past the sequence
-      {
-        const uint4* src = reinterpret_cast<const uint4*>(p.q + row_off);
-        uint8_t* qrow = smem_gen + L::Q_OFF + t * L::Q_BYTES + r * 128;
+      const uint4* src = reinterpret_cast<const uint4*>(p.q + row_off);
+      uint8_t* qrow = smem_gen + L::Q_OFF + qt * L::Q_BYTES + r * 128;
 #pragma unroll
-        for (int c = 0; c < D / 8; ++c) {
-          uint4 v = make_uint4(0, 0, 0, 0);
-          if (valid) v = __ldg(src + c);
-          *reinterpret_cast<uint4*>(qrow + (c >> 3) * L::HALF_BYTES + (((c & 7) ^ (r & 7)) << 4)) = v;
-        }
-        fence_async_smem();
-        mbar_arrive(bar(BAR_Q + t));
+      for (int c = 0; c < D / 8; ++c) {
+        uint4 v = make_uint4(0, 0, 0, 0);
+        if (valid) v = __ldg(src + c);
+        *reinterpret_cast<uint4*>(qrow + (c >> 3) * L::HALF_BYTES + (((c & 7) ^ (r & 7)) << 4)) = v;
       }
-      const uint32_t lane_addr = (uint32_t)((warp & 3) * 32) << 16;
-      const uint32_t s_addr = tmem_S + lane_addr + t * BN;
-      const uint32_t o_addr = tmem_O + lane_addr + t * D;
-      uint8_t* prow = smem_gen + L::P_OFF + t * L::P_BYTES + r * 128;
-      float m_ref = -INFINITY, l_sum = 0.f;
-      for (int jj = 0; jj < nt; ++jj) {
-        mbar_wait(bar(BAR_S + t), jj & 1, abort_flag, p.status);
-        tc_fence_after();
-        uint32_t s[BN];
-        EFIM_TMEM_LD32(s_addr + 0, s + 0);
-        EFIM_TMEM_LD32(s_addr + 32, s + 32);
-        EFIM_TMEM_LD32(s_addr + 64, s + 64);
-        EFIM_TMEM_LD32(s_addr + 96, s + 96);
-        tmem_wait_ld();
-        const int kv0 = (it.tile_begin + jj) * BN;
-        if (__any_sync(0xffffffffu, kv0 + BN > vis)) {
-#pragma unroll
-          for (int c = 0; c < BN; ++c)
-            if (kv0 + c >= vis) s[c] = 0xff800000u;         // -inf
-        }
-        float mx8[8];
-#pragma unroll
-        for (int a = 0; a < 8; ++a) mx8[a] = __uint_as_float(s[a]);
-#pragma unroll
-        for (int c = 8; c < BN; c += 8)
-#pragma unroll
-          for (int a = 0; a < 8; ++a) mx8[a] = fmaxf(mx8[a], __uint_as_float(s[c + a]));
-        const float mx = fmaxf(fmaxf(fmaxf(mx8[0], mx8[1]), fmaxf(mx8[2], mx8[3])),
-                               fmaxf(fmaxf(mx8[4], mx8[5]), fmaxf(mx8[6], mx8[7])));
-        const float m_new = mx * p.scale_log2;
-        // lazy rescale: keep the old reference maximum until it is off by more than 2^8
-        const bool grow = m_new > m_ref + 8.f;
-        if (jj == 0) {
-          m_ref = m_new;
-        } else if (__any_sync(0xffffffffu, grow)) {
-          const float alpha = grow ? ex2(m_ref - m_new) : 1.f;
-          if (grow) m_ref = m_new;
-          l_sum *= alpha;
-#pragma unroll
-          for (int c0 = 0; c0 < D; c0 += 32) {
-            uint32_t o[32];
-            EFIM_TMEM_LD32(o_addr + c0, o);
-            tmem_wait_ld();
-#pragma unroll
-            for (int c = 0; c < 32; ++c) o[c] = __float_as_uint(__uint_as_float(o[c]) * alpha);
-            EFIM_TMEM_ST32(o_addr + c0, o);
-          }
-          tmem_wait_st();
-        }
-        const float m_use = (m_ref == -INFINITY) ? 0.f : m_ref;
-        const float neg_m = -m_use;
-        float ls[4] = {0.f, 0.f, 0.f, 0.f};
-#pragma unroll
-        for (int c16 = 0; c16 < BN / 8; ++c16) {
-          uint32_t w[4];
-#pragma unroll
-          for (int e = 0; e < 4; ++e) {
-            const float p0 = ex2(fmaf(__uint_as_float(s[c16 * 8 + 2 * e]), p.scale_log2, neg_m));
-            const float p1 = ex2(fmaf(__uint_as_float(s[c16 * 8 + 2 * e + 1]), p.scale_log2, neg_m));
-            ls[e] += p0 + p1;
-            w[e] = pack_bf16x2(p0, p1);
-          }
-          *reinterpret_cast<uint4*>(prow + (c16 >> 3) * L::HALF_BYTES + (((c16 & 7) ^ (r & 7)) << 4)) =
-              make_uint4(w[0], w[1], w[2], w[3]);
-        }
-        l_sum += (ls[0] + ls[1]) + (ls[2] + ls[3]);
-        fence_async_smem();
-        tc_fence_before();
-        mbar_arrive(bar(BAR_P + t));
-      }
-      // ---- epilogue: O_t / l -> bf16 output, or fp32 partial + base-2 lse
-      mbar_wait(bar(BAR_O + t), 0, abort_flag, p.status);
+      fence_async_smem();
+      mbar_arrive(bar(BAR_Q + qt));
+    }
+    const uint32_t lane_addr = (uint32_t)((warp & 3) * 32) << 16;
+    const uint32_t s_addr = tmem_S + lane_addr + st * BN;
+    const uint32_t o_addr = tmem_O + lane_addr + st * D;
+    float m_ref = -INFINITY, l_sum = 0.f;
+    for (int k = 0; k < my_cnt; ++k) {
+      mbar_wait(bar(BAR_S + st), k & 1, abort_flag, p.status);
       tc_fence_after();
+      uint32_t s[BN];
+      EFIM_TMEM_LD32(s_addr + 0, s + 0);
+      EFIM_TMEM_LD32(s_addr + 32, s + 32);
+      EFIM_TMEM_LD32(s_addr + 64, s + 64);
+      EFIM_TMEM_LD32(s_addr + 96, s + 96);
+      tmem_wait_ld();
+      const int kv0 = (it.tile_begin + (dual ? k : 2 * k + st)) * BN;
+      if (__any_sync(0xffffffffu, kv0 + BN > vis)) {
+#pragma unroll
+        for (int c = 0; c < BN; ++c)
+          if (kv0 + c >= vis) s[c] = 0xff800000u;           // -inf
+      }
+      float mx8[8];
+#pragma unroll
+      for (int a = 0; a < 8; ++a) mx8[a] = __uint_as_float(s[a]);
+#pragma unroll
+      for (int c = 8; c < BN; c += 8)
+#pragma unroll
+        for (int a = 0; a < 8; ++a) mx8[a] = fmaxf(mx8[a], __uint_as_float(s[c + a]));
+      const float mx = fmaxf(fmaxf(fmaxf(mx8[0], mx8[1]), fmaxf(mx8[2], mx8[3])),
+                             fmaxf(fmaxf(mx8[4], mx8[5]), fmaxf(mx8[6], mx8[7])));
+      const float m_new = mx * p.scale_log2;
+      // lazy rescale: keep the old reference maximum until it is off by more than 2^8
+      const bool grow = m_new > m_ref + 8.f;
+      if (k == 0) {
+        m_ref = m_new;
+      } else if (__any_sync(0xffffffffu, grow)) {
+        const float alpha = grow ? ex2(m_ref - m_new) : 1.f;
+        if (grow) m_ref = m_new;
+        l_sum *= alpha;
+#pragma unroll
+        for (int c0 = 0; c0 < D; c0 += 32) {
+          uint32_t o[32];
+          EFIM_TMEM_LD32(o_addr + c0, o);
+          tmem_wait_ld();
+#pragma unroll
+          for (int c = 0; c < 32; ++c) o[c] = __float_as_uint(__uint_as_float(o[c]) * alpha);
+          EFIM_TMEM_ST32(o_addr + c0, o);
+        }
+      }
+      const float m_use = (m_ref == -INFINITY) ? 0.f : m_ref;
+      const float neg_m = -m_use;
+      float ls[4] = {0.f, 0.f, 0.f, 0.f};
+      // P (bf16 pairs) goes back into the first 64 columns of this stream's S
+#pragma unroll
+      for (int h = 0; h < 2; ++h) {
+        uint32_t w[32];
+#pragma unroll
+        for (int e = 0; e < 32; ++e) {
+          const float p0 = ex2(fmaf(__uint_as_float(s[h * 64 + 2 * e]), p.scale_log2, neg_m));
+          const float p1 = ex2(fmaf(__uint_as_float(s[h * 64 + 2 * e + 1]), p.scale_log2, neg_m));
+          ls[e & 3] += p0 + p1;
+          w[e] = pack_bf16x2(p0, p1);
+        }
+        EFIM_TMEM_ST32(s_addr + h * 32, w);
+      }
+      l_sum += (ls[0] + ls[1]) + (ls[2] + ls[3]);
+      tmem_wait_st();
+      tc_fence_before();
+      mbar_arrive(bar(BAR_P + st));
+    }
+    // ---- epilogue
+    if (my_cnt > 0) {
+      mbar_wait(bar(BAR_O + st), 0, abort_flag, p.status);
+      if (!dual && cnt1 > 0) mbar_wait(bar(BAR_O + (st ^ 1)), 0, abort_flag, p.status);   // ring is quiet
+      tc_fence_after();
+    }
+    float* xbuf = reinterpret_cast<float*>(smem_gen + L::KV_OFF) + r * L::XROW;
+    const bool merge = !dual && cnt1 > 0;
+    if (merge && st == 1) {
+      // stream 1 hands its state to stream 0 through shared memory
+      xbuf[D] = m_ref;
+      xbuf[D + 1] = l_sum;
+#pragma unroll
+      for (int c0 = 0; c0 < D; c0 += 32) {
+        uint32_t o[32];
+        EFIM_TMEM_LD32(o_addr + c0, o);
+        tmem_wait_ld();
+#pragma unroll
+        for (int c = 0; c < 32; c += 4)
+          *reinterpret_cast<uint4*>(xbuf + c0 + c) = make_uint4(o[c], o[c + 1], o[c + 2], o[c + 3]);
+      }
+    }
+    if (merge) asm volatile("bar.sync 1, 256;" ::: "memory");
+    if (my_cnt > 0 && (dual || st == 0)) {
+      float w0 = 1.f, w1 = 0.f;
+      if (merge) {
+        const float m1 = xbuf[D], l1 = xbuf[D + 1];
+        const float M = fmaxf(m_ref, m1);
+        w0 = l_sum > 0.f ? ex2(m_ref - M) : 0.f;
+        w1 = l1 > 0.f ? ex2(m1 - M) : 0.f;
+        l_sum = l_sum * w0 + l1 * w1;
+        m_ref = M;
+      }
       const float inv = l_sum > 0.f ? 1.f / l_sum : 0.f;
       const float lse2 = l_sum > 0.f ? m_ref + log2f(l_sum) : -INFINITY;
+      const float a0 = w0 * inv, a1 = w1 * inv;
       const size_t th = (size_t)(tok0 + i_tok) * p.Hq + (size_t)it.kvh * G + g;
 #pragma unroll
       for (int c0 = 0; c0 < D; c0 += 32) {
         uint32_t o[32];
         EFIM_TMEM_LD32(o_addr + c0, o);
         tmem_wait_ld();
+        float f[32];
+#pragma unroll
+        for (int c = 0; c < 32; ++c) f[c] = __uint_as_float(o[c]) * a0;
+        if (merge) {
+#pragma unroll
+          for (int c = 0; c < 32; c += 4) {
+            const float4 x = *reinterpret_cast<const float4*>(xbuf + c0 + c);
+            f[c] = fmaf(x.x, a1, f[c]);
+            f[c + 1] = fmaf(x.y, a1, f[c + 1]);
+            f[c + 2] = fmaf(x.z, a1, f[c + 2]);
+            f[c + 3] = fmaf(x.w, a1, f[c + 3]);
+          }
+        }
         if (valid) {
           if (it.chunk < 0) {
             uint4* dst = reinterpret_cast<uint4*>(p.out + row_off + c0);
 #pragma unroll
-            for (int c = 0; c < 4; ++c) {
-              uint32_t w[4];
-#pragma unroll
-              for (int e = 0; e < 4; ++e)
-                w[e] = pack_bf16x2(__uint_as_float(o[c * 8 + 2 * e]) * inv, __uint_as_float(o[c * 8 + 2 * e + 1]) * inv);
-              dst[c] = make_uint4(w[0], w[1], w[2], w[3]);
-            }
+            for (int c = 0; c < 4; ++c)
+              dst[c] = make_uint4(pack_bf16x2(f[c * 8], f[c * 8 + 1]), pack_bf16x2(f[c * 8 + 2], f[c * 8 + 3]),
+                                  pack_bf16x2(f[c * 8 + 4], f[c * 8 + 5]), pack_bf16x2(f[c * 8 + 6], f[c * 8 + 7]));
           } else {
             float4* dst = reinterpret_cast<float4*>(p.part_o + (th * p.s_max + it.chunk) * D + c0);
 #pragma unroll
-            for (int c = 0; c < 8; ++c)
-              dst[c] = make_float4(__uint_as_float(o[4 * c]) * inv, __uint_as_float(o[4 * c + 1]) * inv,
-                                   __uint_as_float(o[4 * c + 2]) * inv, __uint_as_float(o[4 * c + 3]) * inv);
+            for (int c = 0; c < 8; ++c) dst[c] = make_float4(f[4 * c], f[4 * c + 1], f[4 * c + 2], f[4 * c + 3]);
           }
         }
       }
@@ -344,8 +398,8 @@ prefill_tc_kernel(const Params p, const __grid_constant__ CUtensorMap map_k, con
           p.part_lse[th * p.s_max + it.chunk] = lse2;
         }
       }
-      tc_fence_before();
     }
+    tc_fence_before();
   } else if (warp == 8) {
     // ============================================================ TMA producer
     const int32_t* bt = p.block_table + (size_t)it.seq * p.max_pages_per_seq;
@@ -385,35 +439,35 @@ prefill_tc_kernel(const Params p, const __grid_constant__ CUtensorMap map_k, con
     // ============================================================ MMA issuer
     constexpr uint32_t IDESC_QK = instr_desc(BN, 0);
     constexpr uint32_t IDESC_PV = instr_desc(D, 1);
-    const uint32_t q_base = smem_base + L::Q_OFF, p_base = smem_base + L::P_OFF, kv_base = smem_base + L::KV_OFF;
-    for (int t = 0; t < nq_active; ++t) mbar_wait(bar(BAR_Q + t), 0, abort_flag, p.status);
+    const uint32_t q_base = smem_base + L::Q_OFF, kv_base = smem_base + L::KV_OFF;
+    mbar_wait(bar(BAR_Q + 0), 0, abort_flag, p.status);
+    if (dual) mbar_wait(bar(BAR_Q + 1), 0, abort_flag, p.status);
     tc_fence_after();
-    // O_t (+)= P_t V for KV tile jv (ring load 2*jv+1)
-    auto issue_pv = [&](int t, int jv) {
-      const uint32_t vb = kv_base + ((2 * jv + 1) % NSTAGE) * L::KV_BYTES;
+    // O_st (+)= P_st V for KV tile n (ring load 2n+1); P comes from TMEM
+    auto issue_pv = [&](int st, int n, uint32_t first) {
+      const uint32_t vb = kv_base + ((2 * n + 1) % NSTAGE) * L::KV_BYTES;
 #pragma unroll
       for (int k = 0; k < BN / 16; ++k) {
-        const uint64_t a = smem_desc(p_base + t * L::P_BYTES + (k >> 2) * L::HALF_BYTES + (k & 3) * 32, 16, 1024);
         const uint64_t b = smem_desc(vb + k * 2048, L::HALF_BYTES, 1024);     // MN-major: LBO = next 64 dims
-        umma_bf16(tmem_O + t * D, a, b, IDESC_PV, (jv > 0 || k > 0) ? 1u : 0u);
+        umma_bf16_ts(tmem_O + st * D, tmem_S + st * BN + k * 8, b, IDESC_PV, (!first || k > 0) ? 1u : 0u);
       }
     };
-    auto issue_qk = [&](int t, int jk) {
-      const uint32_t kb = kv_base + ((2 * jk) % NSTAGE) * L::KV_BYTES;
+    auto issue_qk = [&](int st, int n) {
+      const uint32_t kb = kv_base + ((2 * n) % NSTAGE) * L::KV_BYTES;
+      const uint32_t qb = q_base + (dual ? st : 0) * L::Q_BYTES;
 #pragma unroll
       for (int k = 0; k < D / 16; ++k) {
         const uint32_t off = (k >> 2) * L::HALF_BYTES + (k & 3) * 32;
-        const uint64_t a = smem_desc(q_base + t * L::Q_BYTES + off, 16, 1024);
-        const uint64_t b = smem_desc(kb + off, 16, 1024);
-        umma_bf16(tmem_S + t * BN, a, b, IDESC_QK, k > 0 ? 1u : 0u);
+        umma_bf16(tmem_S + st * BN, smem_desc(qb + off, 16, 1024), smem_desc(kb + off, 16, 1024), IDESC_QK,
+                  k > 0 ? 1u : 0u);
       }
     };
     // V rows past the visible range hold stale or foreign data; P is 0 there but
     // 0 * NaN would poison O, so clear them before the tile is used.
-    auto clear_v_tail = [&](int jv) {
-      const int keys = kv_cap - (it.tile_begin + jv) * BN;
+    auto clear_v_tail = [&](int n) {
+      const int keys = kv_cap - (it.tile_begin + n) * BN;
       if (keys < BN) {
-        uint8_t* vb = smem_gen + L::KV_OFF + ((2 * jv + 1) % NSTAGE) * L::KV_BYTES;
+        uint8_t* vb = smem_gen + L::KV_OFF + ((2 * n + 1) % NSTAGE) * L::KV_BYTES;
         const int first = max(keys, 0);
         const int chunks = (BN - first) * 8 * HALVES;       // 16-byte chunks to clear
         for (int idx = lane; idx < chunks; idx += 32) {
@@ -425,46 +479,38 @@ prefill_tc_kernel(const Params p, const __grid_constant__ CUtensorMap map_k, con
         __syncwarp();
       }
     };
-    for (int jj = 0; jj < nt; ++jj) {
-      if (jj > 0) {
-        const int lv = 2 * (jj - 1) + 1;
-        mbar_wait(bar(BAR_FULL + lv % NSTAGE), (lv / NSTAGE) & 1, abort_flag, p.status);
-        clear_v_tail(jj - 1);
-      }
-      const int lk = 2 * jj;
-      mbar_wait(bar(BAR_FULL + lk % NSTAGE), (lk / NSTAGE) & 1, abort_flag, p.status);
-      tc_fence_after();
-      for (int t = 0; t < nq_active; ++t) {
-        if (jj > 0) {
-          mbar_wait(bar(BAR_P + t), (jj - 1) & 1, abort_flag, p.status);
+    for (int k = 0; k <= cnt0; ++k) {
+#pragma unroll
+      for (int st = 0; st < 2; ++st) {
+        const int my_cnt = st == 0 ? cnt0 : cnt1;
+        if (my_cnt == 0 || k > my_cnt) continue;
+        const bool last_user = !dual || st == 1;            // last stream to touch this K/V tile
+        if (k > 0) {
+          const int n = dual ? k - 1 : 2 * (k - 1) + st;
+          const int lv = 2 * n + 1;
+          mbar_wait(bar(BAR_FULL + lv % NSTAGE), (lv / NSTAGE) & 1, abort_flag, p.status);
+          if (!dual || st == 0) clear_v_tail(n);
+          mbar_wait(bar(BAR_P + st), (k - 1) & 1, abort_flag, p.status);
           tc_fence_after();
           if (lane == 0) {
-            issue_pv(t, jj - 1);
-            if (t == nq_active - 1) tc_commit(bar(BAR_EMPTY + (2 * (jj - 1) + 1) % NSTAGE));   // V[jj-1] is free
+            issue_pv(st, n, k == 1);
+            if (last_user) tc_commit(bar(BAR_EMPTY + lv % NSTAGE));
+            if (k == my_cnt) tc_commit(bar(BAR_O + st));
           }
+          __syncwarp();
         }
-        if (lane == 0) {
-          issue_qk(t, jj);
-          tc_commit(bar(BAR_S + t));
+        if (k < my_cnt) {
+          const int n = dual ? k : 2 * k + st;
+          const int lk = 2 * n;
+          mbar_wait(bar(BAR_FULL + lk % NSTAGE), (lk / NSTAGE) & 1, abort_flag, p.status);
+          tc_fence_after();
+          if (lane == 0) {
+            issue_qk(st, n);
+            tc_commit(bar(BAR_S + st));
+            if (last_user) tc_commit(bar(BAR_EMPTY + lk % NSTAGE));
+          }
+          __syncwarp();
         }
-        __syncwarp();
-      }
-      if (lane == 0) tc_commit(bar(BAR_EMPTY + lk % NSTAGE));                                  // K[jj] is free
-      __syncwarp();
-    }
-    {
-      const int lv = 2 * (nt - 1) + 1;
-      mbar_wait(bar(BAR_FULL + lv % NSTAGE), (lv / NSTAGE) & 1, abort_flag, p.status);
-      clear_v_tail(nt - 1);
-      tc_fence_after();
-      for (int t = 0; t < nq_active; ++t) {
-        mbar_wait(bar(BAR_P + t), (nt - 1) & 1, abort_flag, p.status);
-        tc_fence_after();
-        if (lane == 0) {
-          issue_pv(t, nt - 1);
-          tc_commit(bar(BAR_O + t));
-        }
-        __syncwarp();
       }
     }
     tc_fence_before();
