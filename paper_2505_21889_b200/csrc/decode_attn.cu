@@ -4,8 +4,9 @@
 // products run on fp32 FMAs, the reductions on warp shuffles; no tensor cores.
 //
 // One CTA = (query row, kv head [x group tile], key chunk).  Each of its 4 warps
-// walks whole pages (16 tokens) round-robin.  Inside a warp D/8 lanes share one
-// token row (16 bytes each), so 32/(D/8) tokens are in flight per load.
+// walks whole pages (16 tokens) round-robin, staged into shared memory by bulk
+// copies (one per K page and V page).  Inside a warp D/8 lanes share one token
+// row (16 bytes each), so 32/(D/8) tokens are read per 128-bit shared-memory load.
 #include "decode_attn.cuh"
 
 namespace efim {
@@ -34,16 +35,44 @@ __device__ __forceinline__ void transposed_reduce(float* x, int j) {
   }
 }
 
+// ---- shared-memory staging of whole pages -------------------------------------------
+// One (page, kv head) tile is 16*D*2 contiguous bytes in a pool, so a single bulk copy
+// brings it into shared memory.  Every warp owns a ring of DEC_STAGES stages (K page +
+// V page), keeps DEC_STAGES pages in flight without holding them in registers, and
+// consumes them in order; an mbarrier per stage counts the copied bytes.
+constexpr int DEC_STAGES = 3;
+
+__device__ __forceinline__ uint32_t dec_smem_u32(const void* p) {
+  return static_cast<uint32_t>(__cvta_generic_to_shared(p));
+}
+__device__ __forceinline__ uint32_t dec_mbar_try(uint32_t bar, uint32_t parity) {
+  uint32_t ok;
+  asm volatile(
+      "{\n.reg .pred p;\nmbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\nselp.u32 %0, 1, 0, p;\n}\n"
+      : "=r"(ok)
+      : "r"(bar), "r"(parity)
+      : "memory");
+  return ok;
+}
+__device__ __forceinline__ void dec_bulk_load(uint32_t dst, const void* src, uint32_t bytes, uint32_t bar) {
+  asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];" ::"r"(dst),
+               "l"(src), "r"(bytes), "r"(bar)
+               : "memory");
+}
+
 template <int D, int GT>
 __global__ void __launch_bounds__(128) decode_splitkv_kernel(const DecodeParams p) {
   constexpr int LPT = D / 8;            // lanes sharing one token row
-  constexpr int TPS = 32 / LPT;         // tokens per warp-wide load
-  constexpr int STEPS = 16 / TPS;       // loads per page
+  constexpr int TPS = 32 / LPT;         // tokens per warp-wide 16-byte read
+  constexpr int STEPS = 16 / TPS;       // reads per page
   constexpr int GP = (GT + 1) & ~1;     // heads padded to even
   constexpr int NV = STEPS * GP;        // partial dot products per lane per page
   constexpr int NF = GP / 2;            // finished scores per lane per page
+  constexpr int PAGE_BYTES = 16 * D * 2;
   static_assert(NV / LPT == NF, "reduction leaves GP/2 values per lane");
 
+  extern __shared__ __align__(128) uint8_t dec_ring[];   // [4 warps][DEC_STAGES][K page | V page]
+  __shared__ __align__(8) uint64_t s_bar[4][DEC_STAGES];
   __shared__ float s_p[4][16][GP];      // per warp: probabilities of the current page
   __shared__ float s_m[4][GP], s_l[4][GP];
   __shared__ float s_o[4][GT][D];
@@ -72,124 +101,197 @@ __global__ void __launch_bounds__(128) decode_splitkv_kernel(const DecodeParams 
   const int lane = tid & 31, warp = tid >> 5;
   const int j = lane % LPT, tg = lane / LPT;
 
-  float q[GT][8];
+  // ---- this warp's pages: first_pg, first_pg + 4, ... ; start their copies before anything else
+  const int32_t* bt = p.block_table + (size_t)seq * p.max_pages_per_seq;
+  const int first_pg = (begin >> 4) + warp;
+  const int last_pg = (end - 1) >> 4;
+  const int n_pages = first_pg <= last_pg ? (last_pg - first_pg) / 4 + 1 : 0;
+  uint8_t* ring = dec_ring + warp * (DEC_STAGES * 2 * PAGE_BYTES);
+  if (lane == 0) {
+    for (int sg = 0; sg < DEC_STAGES; ++sg)
+      asm volatile("mbarrier.init.shared::cta.b64 [%0], 1;" ::"r"(dec_smem_u32(&s_bar[warp][sg])) : "memory");
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+  }
+  __syncwarp();
+  // page ids of the next 32 pages of this warp, one per lane (refilled every 32 pages)
+  int pid_cache = (lane < n_pages) ? __ldg(bt + first_pg + 4 * lane) : -1;
+  auto issue = [&](int i) {             // start the copies of this warp's i-th page into stage i % DEC_STAGES
+    const int pid = __shfl_sync(0xffffffffu, pid_cache, i & 31);
+    const bool ok = pid >= 0 && pid < p.num_pages;
+    if (lane == 0) {
+      const uint32_t bar = dec_smem_u32(&s_bar[warp][i % DEC_STAGES]);
+      if (ok) {
+        const uint32_t dst = dec_smem_u32(ring + (i % DEC_STAGES) * 2 * PAGE_BYTES);
+        const size_t off = ((size_t)pid * p.Hkv + kvh) * 16 * D;
+        asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(2 * PAGE_BYTES) : "memory");
+        dec_bulk_load(dst, p.k_pool + off, PAGE_BYTES, bar);
+        dec_bulk_load(dst + PAGE_BYTES, p.v_pool + off, PAGE_BYTES, bar);
+      } else {
+        asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");   // nothing to copy
+        if (p.status) atomicOr(p.status, EFIM_DEV_BAD_PAGE);
+      }
+    }
+    return ok;
+  };
+  uint32_t ok_bits = 0;                 // which of the in-flight pages are valid (bit = stage)
+#pragma unroll
+  for (int i = 0; i < DEC_STAGES; ++i)
+    if (i < n_pages && issue(i)) ok_bits |= 1u << i;
+
+  // q and o as packed fp32 pairs (dims 2e, 2e+1): the inner products and the P V
+  // update run on two-wide FMAs
+  uint64_t q2[GT][4];
 #pragma unroll
   for (int g = 0; g < GT; ++g) {
     if (g < ng) {
       const uint4 w = __ldg(reinterpret_cast<const uint4*>(p.q + ((size_t)r * p.Hq + head0 + g) * D) + j);
       const uint32_t* u = reinterpret_cast<const uint32_t*>(&w);
 #pragma unroll
-      for (int e = 0; e < 4; ++e) {
-        q[g][2 * e] = bf16lo(u[e]) * p.scale_log2;
-        q[g][2 * e + 1] = bf16hi(u[e]) * p.scale_log2;
-      }
+      for (int e = 0; e < 4; ++e) q2[g][e] = pack2(bf16lo(u[e]) * p.scale_log2, bf16hi(u[e]) * p.scale_log2);
     } else {
 #pragma unroll
-      for (int e = 0; e < 8; ++e) q[g][e] = 0.f;
+      for (int e = 0; e < 4; ++e) q2[g][e] = 0ull;
     }
   }
-  float o[GT][8];
+  uint64_t o2[GT][4];
 #pragma unroll
   for (int g = 0; g < GT; ++g)
 #pragma unroll
-    for (int e = 0; e < 8; ++e) o[g][e] = 0.f;
+    for (int e = 0; e < 4; ++e) o2[g][e] = 0ull;
   float m_run[GP], l_part[NF];
 #pragma unroll
   for (int g = 0; g < GP; ++g) m_run[g] = -INFINITY;
 #pragma unroll
   for (int i = 0; i < NF; ++i) l_part[i] = 0.f;
 
-  const int32_t* bt = p.block_table + (size_t)seq * p.max_pages_per_seq;
   const int odd = j & 1;
   const int st_mine = j >> 1;                   // step whose scores this lane ends up with
+  bool gave_up = false;
 
-  for (int pg = (begin >> 4) + warp; (pg << 4) < end; pg += 4) {
-    const int page = __ldg(bt + pg);
-    if (page < 0 || page >= p.num_pages) {      // warp-uniform
-      if (lane == 0 && p.status) atomicOr(p.status, EFIM_DEV_BAD_PAGE);
-      continue;
-    }
-    const size_t base = (((size_t)page * p.Hkv + kvh) * 16 + tg) * D + j * 8;
-    uint4 kreg[STEPS], vreg[STEPS];
-#pragma unroll
-    for (int st = 0; st < STEPS; ++st) kreg[st] = ldg_stream(p.k_pool + base + (size_t)st * TPS * D);
-#pragma unroll
-    for (int st = 0; st < STEPS; ++st) vreg[st] = ldg_stream(p.v_pool + base + (size_t)st * TPS * D);
-
-    // ---- scores: partial dot products over this lane's 8 dims, then the cross-lane sum
-    float x[NV];
-#pragma unroll
-    for (int st = 0; st < STEPS; ++st) {
-      const uint32_t* u = reinterpret_cast<const uint32_t*>(&kreg[st]);
-      float kf[8];
-#pragma unroll
-      for (int e = 0; e < 4; ++e) { kf[2 * e] = bf16lo(u[e]); kf[2 * e + 1] = bf16hi(u[e]); }
-#pragma unroll
-      for (int g = 0; g < GP; ++g) {
-        float acc = 0.f;
-        if (g < GT) {
-#pragma unroll
-          for (int e = 0; e < 8; ++e) acc = fmaf(q[g][e], kf[e], acc);
-        }
-        x[st * GP + g] = acc;
-      }
-    }
-    transposed_reduce<NV, LPT>(x, j);
-    // lane j now holds, for token (st_mine*TPS + tg) of the page, heads odd*NF + i
-    const int tok_in_page = st_mine * TPS + tg;
-    const bool visible = (pg << 4) + tok_in_page < end;
-    float sc[NF], mx[NF];
-#pragma unroll
-    for (int i = 0; i < NF; ++i) { sc[i] = visible ? x[i] : -INFINITY; mx[i] = sc[i]; }
-#pragma unroll
-    for (int off = 2; off < 32; off <<= 1)
-#pragma unroll
-      for (int i = 0; i < NF; ++i) mx[i] = fmaxf(mx[i], __shfl_xor_sync(0xffffffffu, mx[i], off));
-    float alpha[GP], mine[NF], alpha_mine[NF];
-#pragma unroll
-    for (int i = 0; i < NF; ++i) {
-      const float other = __shfl_xor_sync(0xffffffffu, mx[i], 1);
-      const float m_lo = odd ? other : mx[i];       // head i
-      const float m_hi = odd ? mx[i] : other;       // head NF + i
-      const float n_lo = fmaxf(m_run[i], m_lo), n_hi = fmaxf(m_run[NF + i], m_hi);
-      alpha[i] = exp2f(m_run[i] - n_lo);
-      alpha[NF + i] = exp2f(m_run[NF + i] - n_hi);
-      m_run[i] = n_lo;
-      m_run[NF + i] = n_hi;
-      mine[i] = odd ? n_hi : n_lo;
-      alpha_mine[i] = odd ? alpha[NF + i] : alpha[i];
-    }
-#pragma unroll
-    for (int i = 0; i < NF; ++i) {
-      const float pr = exp2f(sc[i] - mine[i]);      // masked: exp2(-inf) = 0
-      l_part[i] = fmaf(l_part[i], alpha_mine[i], pr);
-      s_p[warp][tok_in_page][odd * NF + i] = pr;
-    }
-    __syncwarp();
-    // ---- values
-#pragma unroll
-    for (int g = 0; g < GT; ++g)
-#pragma unroll
-      for (int e = 0; e < 8; ++e) o[g][e] *= alpha[g];
-#pragma unroll
-    for (int st = 0; st < STEPS; ++st) {
-      const int tp = st * TPS + tg;
-      if ((pg << 4) + tp < end) {                   // never touch slots past the context
-        const uint32_t* u = reinterpret_cast<const uint32_t*>(&vreg[st]);
-        float vf[8];
-#pragma unroll
-        for (int e = 0; e < 4; ++e) { vf[2 * e] = bf16lo(u[e]); vf[2 * e + 1] = bf16hi(u[e]); }
-#pragma unroll
-        for (int g = 0; g < GT; ++g) {
-          const float pr = s_p[warp][tp][g];
-#pragma unroll
-          for (int e = 0; e < 8; ++e) o[g][e] = fmaf(pr, vf[e], o[g][e]);
+  for (int i = 0; i < n_pages; ++i) {
+    const int pg = first_pg + 4 * i;
+    const int sg = i % DEC_STAGES;
+    const bool page_ok = (ok_bits >> sg) & 1u;
+    // ---- wait for the stage (bounded: ~2 s, then flag and stop)
+    {
+      const uint32_t bar = dec_smem_u32(&s_bar[warp][sg]);
+      const uint32_t parity = (i / DEC_STAGES) & 1;
+      if (!dec_mbar_try(bar, parity)) {
+        unsigned long long t0, t1;
+        asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t0));
+        uint32_t spins = 0;
+        while (!dec_mbar_try(bar, parity)) {
+          if ((++spins & 1023u) == 0) {
+            asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t1));
+            if (t1 - t0 > 2000000000ull) { gave_up = true; break; }
+          }
         }
       }
+      gave_up = __any_sync(0xffffffffu, gave_up);
+      if (gave_up) {
+        if (lane == 0 && p.status) atomicOr(p.status, EFIM_DEV_TIMEOUT);
+        break;
+      }
     }
-    __syncwarp();
+    if (page_ok) {
+      const uint8_t* kst = ring + sg * 2 * PAGE_BYTES + (tg * D + j * 8) * 2;
+      const uint8_t* vst = kst + PAGE_BYTES;
+      // ---- scores: partial dot products over this lane's 8 dims, then the cross-lane sum
+      float x[NV];
+#pragma unroll
+      for (int st = 0; st < STEPS; ++st) {
+        const uint4 kv = *reinterpret_cast<const uint4*>(kst + st * TPS * D * 2);
+        const uint32_t* u = reinterpret_cast<const uint32_t*>(&kv);
+        uint64_t k2[4];
+#pragma unroll
+        for (int e = 0; e < 4; ++e) k2[e] = pack2(bf16lo(u[e]), bf16hi(u[e]));
+#pragma unroll
+        for (int g = 0; g < GP; ++g) {
+          float acc = 0.f;
+          if (g < GT) {
+            uint64_t a2 = 0ull;
+#pragma unroll
+            for (int e = 0; e < 4; ++e) a2 = ffma2(q2[g][e], k2[e], a2);
+            float lo, hi;
+            unpack2(a2, lo, hi);
+            acc = lo + hi;
+          }
+          x[st * GP + g] = acc;
+        }
+      }
+      transposed_reduce<NV, LPT>(x, j);
+      // lane j now holds, for token (st_mine*TPS + tg) of the page, heads odd*NF + i
+      const int tok_in_page = st_mine * TPS + tg;
+      const bool visible = (pg << 4) + tok_in_page < end;
+      float sc[NF], mx[NF];
+#pragma unroll
+      for (int a = 0; a < NF; ++a) { sc[a] = visible ? x[a] : -INFINITY; mx[a] = sc[a]; }
+#pragma unroll
+      for (int off = 2; off < 32; off <<= 1)
+#pragma unroll
+        for (int a = 0; a < NF; ++a) mx[a] = fmaxf(mx[a], __shfl_xor_sync(0xffffffffu, mx[a], off));
+      float alpha[GP], mine[NF], alpha_mine[NF];
+#pragma unroll
+      for (int a = 0; a < NF; ++a) {
+        const float other = __shfl_xor_sync(0xffffffffu, mx[a], 1);
+        const float m_lo = odd ? other : mx[a];       // head a
+        const float m_hi = odd ? mx[a] : other;       // head NF + a
+        const float n_lo = fmaxf(m_run[a], m_lo), n_hi = fmaxf(m_run[NF + a], m_hi);
+        alpha[a] = exp2f(m_run[a] - n_lo);
+        alpha[NF + a] = exp2f(m_run[NF + a] - n_hi);
+        m_run[a] = n_lo;
+        m_run[NF + a] = n_hi;
+        mine[a] = odd ? n_hi : n_lo;
+        alpha_mine[a] = odd ? alpha[NF + a] : alpha[a];
+      }
+#pragma unroll
+      for (int a = 0; a < NF; ++a) {
+        const float pr = exp2f(sc[a] - mine[a]);      // masked: exp2(-inf) = 0
+        l_part[a] = fmaf(l_part[a], alpha_mine[a], pr);
+        s_p[warp][tok_in_page][odd * NF + a] = pr;
+      }
+      __syncwarp();
+      // ---- values
+#pragma unroll
+      for (int g = 0; g < GT; ++g) {
+        const uint64_t al2 = pack2(alpha[g], alpha[g]);
+#pragma unroll
+        for (int e = 0; e < 4; ++e) o2[g][e] = fmul2(o2[g][e], al2);
+      }
+#pragma unroll
+      for (int st = 0; st < STEPS; ++st) {
+        const int tp = st * TPS + tg;
+        if ((pg << 4) + tp < end) {                   // never touch slots past the context
+          const uint4 vv = *reinterpret_cast<const uint4*>(vst + st * TPS * D * 2);
+          const uint32_t* u = reinterpret_cast<const uint32_t*>(&vv);
+          uint64_t v2[4];
+#pragma unroll
+          for (int e = 0; e < 4; ++e) v2[e] = pack2(bf16lo(u[e]), bf16hi(u[e]));
+#pragma unroll
+          for (int g = 0; g < GT; ++g) {
+            const float pr = s_p[warp][tp][g];
+            const uint64_t pr2 = pack2(pr, pr);
+#pragma unroll
+            for (int e = 0; e < 4; ++e) o2[g][e] = ffma2(pr2, v2[e], o2[g][e]);
+          }
+        }
+      }
+    }
+    __syncwarp();                                     // everyone is done with the stage and with s_p
+    // ---- refill the stage with the page DEC_STAGES ahead
+    const int nxt = i + DEC_STAGES;
+    if (nxt < n_pages) {
+      if ((nxt & 31) == 0) pid_cache = (nxt + lane < n_pages) ? __ldg(bt + first_pg + 4 * (nxt + lane)) : -1;
+      ok_bits &= ~(1u << sg);
+      if (issue(nxt)) ok_bits |= 1u << sg;
+    }
   }
 
+  float o[GT][8];
+#pragma unroll
+  for (int g = 0; g < GT; ++g)
+#pragma unroll
+    for (int e = 0; e < 4; ++e) unpack2(o2[g][e], o[g][2 * e], o[g][2 * e + 1]);
   // ---- fold the token groups of the warp, then the 4 warps
 #pragma unroll
   for (int off = LPT; off < 32; off <<= 1)
@@ -298,15 +400,26 @@ DecodePlan plan_decode(int rows, int Hq, int Hkv, int D, int max_len) {
   return pl;
 }
 
+template <int D, int GT>
+static efim_status launch_split(const DecodeParams& p, dim3 grid, cudaStream_t s) {
+  constexpr int ring_bytes = 4 * DEC_STAGES * 2 * 16 * D * 2;      // 4 warps x stages x (K page + V page)
+  EFIM_CUDA_TRY(cudaFuncSetAttribute(decode_splitkv_kernel<D, GT>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                     ring_bytes));
+  decode_splitkv_kernel<D, GT><<<grid, 128, ring_bytes, s>>>(p);
+  return EFIM_OK;
+}
+
 template <int D>
 static efim_status launch_decode_d(const DecodeParams& p, const DecodePlan& pl, cudaStream_t s) {
   dim3 grid(p.R, p.Hkv * pl.gsplit, pl.n_chunks);
+  efim_status st;
   switch (pl.group_tile) {
-    case 1: decode_splitkv_kernel<D, 1><<<grid, 128, 0, s>>>(p); break;
-    case 2: decode_splitkv_kernel<D, 2><<<grid, 128, 0, s>>>(p); break;
-    case 3: decode_splitkv_kernel<D, 3><<<grid, 128, 0, s>>>(p); break;
-    default: decode_splitkv_kernel<D, 4><<<grid, 128, 0, s>>>(p); break;
+    case 1: st = launch_split<D, 1>(p, grid, s); break;
+    case 2: st = launch_split<D, 2>(p, grid, s); break;
+    case 3: st = launch_split<D, 3>(p, grid, s); break;
+    default: st = launch_split<D, 4>(p, grid, s); break;
   }
+  if (st != EFIM_OK) return st;
   EFIM_CUDA_TRY(cudaGetLastError());
   if (pl.n_chunks > 1) {
     const unsigned blocks = (unsigned)(((size_t)p.R * p.Hq + 3) / 4);
