@@ -91,9 +91,12 @@ class DeviceWorkload:
         return torch_to_bits(pool[idx])
 
     # ---- oracle on a subset of sequences ------------------------------------
-    def oracle_turn(self, seqs=None, sm_scale=None):
+    def oracle_turn(self, seqs=None, sm_scale=None, windows=None):
         """Run the oracle's kv_append + append_prefill_attention for `seqs`.
-        Returns dict with rotated q bits, pools (compact), block table, o, lse, row index."""
+        Returns dict with rotated q bits, pools (compact), block table, o, lse, row index.
+        `windows` = list of (first_token, count) per sequence restricts the attention rows
+        to those new tokens (the cache update is still done for all of them); by the reuse
+        identity this is the oracle called with cached_len + first_token."""
         w = self.w
         kp, vp, bt, seqs = w.compact_host_pool(seqs)
         ind = w.q_indptr
@@ -102,6 +105,17 @@ class DeviceWorkload:
         new = w.new_len[seqs]
         q_rot = orc.kv_append(kp, vp, bt, cached, new, self.q_bits[rows], self.k_bits[rows], self.v_bits[rows],
                               w.rope_base, self.interleaved, use_rope=self.rope is not None)
-        o, lse = orc.append_prefill_attention(q_rot, kp, vp, bt, cached, new, w.num_q_heads, sm_scale)
+        attn_rows = rows
+        if windows is None:
+            o, lse = orc.append_prefill_attention(q_rot, kp, vp, bt, cached, new, w.num_q_heads, sm_scale)
+        else:
+            starts = np.concatenate([[0], np.cumsum(new)])[:-1]
+            first = np.array([f for f, _ in windows], np.int64)
+            cnt = np.array([min(c, int(n) - f) for (f, c), n in zip(windows, new)], np.int64)
+            local = np.concatenate([np.arange(starts[i] + first[i], starts[i] + first[i] + cnt[i])
+                                    for i in range(len(seqs))]).astype(np.int64)
+            o, lse = orc.append_prefill_attention(q_rot[local], kp, vp, bt, cached + first, cnt, w.num_q_heads,
+                                                  sm_scale)
+            attn_rows = rows[local]
         return dict(q_rot=q_rot, k_pool=kp, v_pool=vp, bt=bt, seqs=seqs, rows=rows, o=o, lse=lse,
-                    cached=cached, new=new)
+                    cached=cached, new=new, attn_rows=attn_rows)

@@ -1,0 +1,100 @@
+"""Parity at the full sizes of the five configs, in the launch configuration bench.py
+times.  The GPU processes the whole batch; the oracle recomputes sampled sequences
+(and, for the long FIM-miss rows, sampled token windows) from the same seeded bytes."""
+import numpy as np
+import pytest
+import torch
+
+import paper_2505_21889_b200 as efim
+from efim_synth import make_workload
+from oracle import efim_oracle as orc
+
+pytestmark = pytest.mark.gpu
+
+
+def _run_turn(w, seqs, windows=None):
+    import tests.gpu_harness as H
+    dw = H.DeviceWorkload(w)
+    dw.gpu_kv_append()
+    dw.gpu_prefill()
+    torch.cuda.synchronize()
+    assert int(dw.status.item()) == 0
+    ref = dw.oracle_turn(seqs, windows=windows)
+    for r, s in enumerate(ref["seqs"]):
+        pg = w.pages_of(s, int(w.cached_len[s] + w.new_len[s]))
+        assert np.array_equal(dw.pages_from_device("v", pg), ref["v_pool"][ref["bt"][r, :len(pg)]])
+        H.assert_rope_close(dw.pages_from_device("k", pg), ref["k_pool"][ref["bt"][r, :len(pg)]], f"{w.name} K pages")
+    H.assert_rope_close(H.torch_to_bits(dw.q)[ref["rows"]], ref["q_rot"], f"{w.name} q")
+    H.assert_attn_close(H.torch_to_bits(dw.out)[ref["attn_rows"]], ref["o"], f"{w.name} full size")
+    assert np.abs(dw.lse.cpu().numpy()[ref["attn_rows"]] - ref["lse"]).max() <= H.LSE_TOL
+    # every output of the batch is finite (also the rows the oracle did not recompute)
+    assert torch.isfinite(dw.out.float()).all()
+    return dw, ref
+
+
+def test_cfg2_full_sampled_sequences():
+    w = make_workload("cfg2")
+    order = np.argsort(w.cached_len + w.new_len)
+    _run_turn(w, sorted([int(order[0]), int(order[-1]), int(order[7])]))
+
+
+def test_cfg3_full_sampled_rows():
+    w = make_workload("cfg3")
+    pre = np.where(~w.decode_rows)[0]
+    dec = np.where(w.decode_rows)[0]
+    L = w.cached_len + w.new_len
+    picks = [int(pre[np.argmin(L[pre])]), int(pre[np.argmax(w.new_len[pre])]), int(dec[np.argmax(L[dec])]),
+             int(dec[0])]
+    _run_turn(w, sorted(set(picks)))
+
+
+def test_cfg4a_full_one_sequence():
+    _run_turn(make_workload("cfg4a"), [3])
+
+
+@pytest.mark.parametrize("name", ["cfg4b", "cfg4b_3072"])
+def test_cfg4b_full_token_windows(name):
+    w = make_workload(name)
+    n = int(w.new_len[5])
+    # three windows of the recomputed suffix: start, middle (across a tile edge), end
+    for first in (0, n // 2 - 24, n - 48):
+        _run_turn(w, [5], windows=[(first, 48)])
+
+
+def test_cfg5_full_decode_steps_sampled():
+    import tests.gpu_harness as H
+    w = make_workload("cfg5")
+    dw = H.DeviceWorkload(w)
+    ctx_all = w.cached_len.astype(np.int32).copy()
+    order = np.argsort(ctx_all)
+    seqs = sorted([int(order[0]), int(order[-1]), int(order[100])])
+    kp, vp, bt, seqs = w.compact_host_pool(seqs)
+    B = w.batch
+    steps = 3
+    max_ctx = int(ctx_all.max()) + w.decode_steps
+    ws = torch.empty(max(efim.efim_decode_workspace_bytes(dw.cache, B, max_ctx), 256), dtype=torch.uint8, device="cuda")
+    one_all = np.ones(B, np.int32)
+    one = np.ones(len(seqs), np.int32)
+    ctx = ctx_all[seqs].copy()
+    for step in range(steps):
+        q, k, v = w.decode_qkv(step)
+        q_rot = orc.kv_append(kp, vp, bt, ctx, one, q[seqs], k[seqs], v[seqs], w.rope_base)
+        sb = efim.Batch(ctx_all, one_all, dw.batch.d_block_table)
+        ctx_all = ctx_all + 1
+        ctx = ctx + 1
+        o, lse = orc.decode_attention(q_rot, kp, vp, bt, ctx, w.num_q_heads)
+        dq, dk, dv = H.bits_to_torch(q), H.bits_to_torch(k), H.bits_to_torch(v)
+        efim.efim_kv_append(dw.cache, sb, dw.rope, dq, dk, dv, dw.status)
+        out = torch.empty_like(dq)
+        lse_d = torch.empty((B, w.num_q_heads), dtype=torch.float32, device="cuda")
+        efim.efim_decode_attn(dw.cache, B, torch.from_numpy(ctx_all).cuda(), max_ctx, dw.batch.d_block_table, dq, out,
+                              lse_d, 0.0, ws, dw.status)
+        torch.cuda.synchronize()
+        assert int(dw.status.item()) == 0
+        H.assert_attn_close(H.torch_to_bits(out)[seqs], o, f"cfg5 full decode step {step}")
+        assert np.abs(lse_d.cpu().numpy()[seqs] - lse).max() <= H.LSE_TOL
+        assert torch.isfinite(out.float()).all()
+    for r, s in enumerate(seqs):
+        pg = w.pages_of(s, int(ctx_all[s]))[-2:]
+        want = vp[bt[r, len(w.pages_of(s, int(ctx_all[s]))) - 2: len(w.pages_of(s, int(ctx_all[s])))]]
+        assert np.array_equal(dw.pages_from_device("v", pg), want)
