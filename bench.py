@@ -315,11 +315,10 @@ def run_native(args):
         if has_decode:
             h_dout.copy_(dout.view(torch.int16), non_blocking=True)
 
-    # launches of our kernels per step: kv_append 1; prefill = row expansion + split-KV (+ merge);
-    # decode = split-KV (+ merge when the context is cut into chunks)
-    launches = 1 + 3
+    # launches of our kernels per step, as the library plans them
+    launches = 1 + efim.efim_prefill_launch_count(cache, batch)
     if has_decode:
-        launches += 1 + (2 if dec_ws_bytes > 0 else 1)
+        launches += 1 + efim.efim_decode_launch_count(cache, B, max_ctx)
 
     def barrier():
         if dist is not None:

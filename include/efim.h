@@ -146,6 +146,11 @@ efim_status efim_append_prefill_attn(const efim_cache_desc* cache, const efim_ba
  * ctx_len[s] == 0 gives out = 0, lse = -inf.
  */
 size_t efim_decode_workspace_bytes(const efim_cache_desc* cache, int32_t batch, int32_t max_ctx_len);
+/* Number of kernels the corresponding call enqueues for these arguments (the main
+ * kernel, plus a merge kernel when the key range is split); 0 for invalid arguments.
+ * Planning queries for profiling and launch accounting; they launch nothing. */
+int32_t efim_prefill_launch_count(const efim_cache_desc* cache, const efim_batch_desc* batch);
+int32_t efim_decode_launch_count(const efim_cache_desc* cache, int32_t batch, int32_t max_ctx_len);
 efim_status efim_decode_attn(const efim_cache_desc* cache, int32_t batch,
                              const int32_t* d_ctx_len, int32_t max_ctx_len,
                              const int32_t* d_block_table, int32_t max_pages_per_seq,

@@ -36,7 +36,8 @@ class _RopeDesc(Structure):
 EXPORTS = ("efim_strerror", "efim_version", "efim_rope_table_build", "efim_kv_append",
            "efim_prefill_workspace_bytes", "efim_append_prefill_attn",
            "efim_decode_workspace_bytes", "efim_decode_attn",
-           "efim_decode_static_scratch_bytes", "efim_decode_attn_static")
+           "efim_decode_static_scratch_bytes", "efim_decode_attn_static",
+           "efim_prefill_launch_count", "efim_decode_launch_count")
 
 
 def library_path() -> str:
@@ -72,6 +73,10 @@ def load_library():
     lib.efim_decode_attn.argtypes = [POINTER(_CacheDesc), c_int32, c_void_p, c_int32, c_void_p, c_int32,
                                      c_void_p, c_void_p, c_void_p, c_float, c_void_p, c_size_t,
                                      c_void_p, c_void_p]
+    lib.efim_prefill_launch_count.restype = c_int32
+    lib.efim_prefill_launch_count.argtypes = [POINTER(_CacheDesc), POINTER(_BatchDesc)]
+    lib.efim_decode_launch_count.restype = c_int32
+    lib.efim_decode_launch_count.argtypes = [POINTER(_CacheDesc), c_int32, c_int32]
     lib.efim_decode_static_scratch_bytes.restype = c_size_t
     lib.efim_decode_static_scratch_bytes.argtypes = []
     lib.efim_decode_attn_static.restype = ctypes.c_int
@@ -218,3 +223,11 @@ def efim_decode_attn_static(cache: Cache, batch: int, d_ctx_len, max_ctx_len, d_
                                                 _stream_ptr(stream))
     if st != 0:
         raise EfimError(st, "efim_decode_attn_static")
+
+
+def efim_prefill_launch_count(cache: Cache, batch: Batch) -> int:
+    return int(load_library().efim_prefill_launch_count(ctypes.byref(cache.desc), ctypes.byref(batch.desc)))
+
+
+def efim_decode_launch_count(cache: Cache, batch: int, max_ctx_len: int) -> int:
+    return int(load_library().efim_decode_launch_count(ctypes.byref(cache.desc), batch, max_ctx_len))

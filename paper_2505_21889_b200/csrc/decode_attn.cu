@@ -444,6 +444,13 @@ extern "C" size_t efim_decode_workspace_bytes(const efim_cache_desc* cache, int3
   return pl.part_o_bytes + pl.part_lse_bytes;
 }
 
+extern "C" int32_t efim_decode_launch_count(const efim_cache_desc* cache, int32_t batch, int32_t max_ctx_len) {
+  if (efim::check_cache(cache) != EFIM_OK || batch <= 0) return 0;
+  const efim::DecodePlan pl = efim::plan_decode(batch, cache->num_q_heads, cache->num_kv_heads, cache->head_dim,
+                                                max_ctx_len);
+  return pl.n_chunks > 1 ? 2 : 1;
+}
+
 extern "C" efim_status efim_decode_attn(const efim_cache_desc* cache, int32_t batch, const int32_t* d_ctx_len,
                                         int32_t max_ctx_len, const int32_t* d_block_table,
                                         int32_t max_pages_per_seq, const void* d_q, void* d_out, float* d_lse,

@@ -11,6 +11,13 @@ extern "C" size_t efim_prefill_workspace_bytes(const efim_cache_desc* cache, con
   return efim::pf::make_plan(cache, batch, nullptr, nullptr).total();
 }
 
+extern "C" int32_t efim_prefill_launch_count(const efim_cache_desc* cache, const efim_batch_desc* batch) {
+  if (efim::check_cache(cache) != EFIM_OK || efim::check_batch(cache, batch, true) != EFIM_OK) return 0;
+  if (batch->batch == 0 || batch->total_new_tokens == 0) return 0;
+  const efim::pf::Plan pl = efim::pf::make_plan(cache, batch, nullptr, nullptr);
+  return pl.n_items == 0 ? 0 : (pl.s_max > 1 ? 2 : 1);
+}
+
 extern "C" efim_status efim_append_prefill_attn(const efim_cache_desc* cache, const efim_batch_desc* batch,
                                                 const void* d_q, void* d_out, float* d_lse, float sm_scale,
                                                 void* d_workspace, size_t workspace_bytes, int32_t* d_status,

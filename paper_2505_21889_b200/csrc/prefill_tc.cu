@@ -7,7 +7,8 @@
 // tiles of 128 keys (8 pages):
 //   warp 8    TMA producer: walks the block table, one tiled bulk-tensor copy per
 //             (page, 64-dim half) into a 5-entry shared-memory ring (128B swizzle)
-//   warp 9    issues tcgen05.mma: S_t = Q_t K^T into TMEM, then O_t += P_t V (P from TMEM)
+//   warp 10   issues the tcgen05.mma for S_t = Q_t K^T into TMEM
+//   warp 9    issues the tcgen05.mma for O_t += P_t V (P read from TMEM)
 //   warps 0-7 two softmax groups, one per query tile, one TMEM lane (row) per thread:
 //             S from TMEM, mask, running max with lazy rescale, exp2, P (bf16) back to
 //             TMEM over S, final normalisation and store
@@ -158,7 +159,11 @@ struct Smem {
   static_assert(BM * XROW * 4 <= NSTAGE * KV_BYTES, "exchange buffer must fit in the ring");
 };
 // barrier slots (8 bytes each) inside the BAR_OFF block
-enum { BAR_Q = 0, BAR_S = 2, BAR_P = 4, BAR_O = 6, BAR_FULL = 8, BAR_EMPTY = 8 + NSTAGE, BAR_COUNT = 8 + 2 * NSTAGE };
+// (P has two barriers per stream: keys 0-63 and 64-127 of a tile are handed over separately)
+enum {
+  BAR_Q = 0, BAR_S = 2, BAR_P = 4, BAR_O = 8, BAR_PVI = 10, BAR_FULL = 12, BAR_EMPTY = 12 + NSTAGE,
+  BAR_COUNT = 12 + 2 * NSTAGE
+};
 
 // Two softmax groups ("streams") run per CTA.  With more than 128 rows, stream t
 // owns query tile t and both walk every KV tile.  With 128 rows or fewer there is
@@ -197,8 +202,10 @@ prefill_tc_kernel(const Params p, const __grid_constant__ CUtensorMap map_k, con
     for (int t = 0; t < NQ; ++t) {
       mbar_init(bar(BAR_Q + t), BM);
       mbar_init(bar(BAR_S + t), 1);
-      mbar_init(bar(BAR_P + t), BM);
+      mbar_init(bar(BAR_P + 2 * t), BM);
+      mbar_init(bar(BAR_P + 2 * t + 1), BM);
       mbar_init(bar(BAR_O + t), 1);
+      mbar_init(bar(BAR_PVI + t), 1);
     }
     for (int s = 0; s < NSTAGE; ++s) {
       mbar_init(bar(BAR_FULL + s), 1);
@@ -301,10 +308,10 @@ prefill_tc_kernel(const Params p, const __grid_constant__ CUtensorMap map_k, con
           EFIM_TMEM_ST32(o_addr + c0, o);
         }
       }
-      const float m_use = (m_ref == -INFINITY) ? 0.f : m_ref;
-      const float neg_m = -m_use;
+      const float neg_m = (m_ref == -INFINITY) ? 0.f : -m_ref;
       float ls[4] = {0.f, 0.f, 0.f, 0.f};
-      // P (bf16 pairs) goes back into the first 64 columns of this stream's S
+      // P (bf16 pairs) goes back into the first 64 columns of this stream's S, in two
+      // halves of 64 keys, so the PV MMAs of the first half are issued under the second
 #pragma unroll
       for (int h = 0; h < 2; ++h) {
         uint32_t w[32];
@@ -316,11 +323,11 @@ prefill_tc_kernel(const Params p, const __grid_constant__ CUtensorMap map_k, con
           w[e] = pack_bf16x2(p0, p1);
         }
         EFIM_TMEM_ST32(s_addr + h * 32, w);
+        tmem_wait_st();
+        tc_fence_before();
+        mbar_arrive(bar(BAR_P + 2 * st + h));
       }
       l_sum += (ls[0] + ls[1]) + (ls[2] + ls[3]);
-      tmem_wait_st();
-      tc_fence_before();
-      mbar_arrive(bar(BAR_P + st));
     }
     // ---- epilogue
     if (my_cnt > 0) {
@@ -435,31 +442,42 @@ prefill_tc_kernel(const Params p, const __grid_constant__ CUtensorMap map_k, con
         for (int spin = 0; spin < (1 << 20) && !mbar_try(b, par); ++spin) {}
       }
     }
-  } else if (warp == 9) {
-    // ============================================================ MMA issuer
+  } else if (warp == 9 || warp == 10) {
+    // ============================================================ MMA issuers
+    // Issuing an MMA costs its thread about as long as the tensor core needs to run it,
+    // so the work is split: warp 9 issues the PV MMAs of both streams, warp 10 the QK
+    // MMAs.  QK(k+1) of a stream overwrites the columns P(k) is read from, so warp 10
+    // issues it only after warp 9 has issued PV(k) (barrier PVI, tcgen05 fences on both
+    // sides); the tensor core runs them in that order.
+    const bool pv_role = warp == 9;
     constexpr uint32_t IDESC_QK = instr_desc(BN, 0);
     constexpr uint32_t IDESC_PV = instr_desc(D, 1);
     const uint32_t q_base = smem_base + L::Q_OFF, kv_base = smem_base + L::KV_OFF;
     mbar_wait(bar(BAR_Q + 0), 0, abort_flag, p.status);
     if (dual) mbar_wait(bar(BAR_Q + 1), 0, abort_flag, p.status);
     tc_fence_after();
-    // O_st (+)= P_st V for KV tile n (ring load 2n+1); P comes from TMEM
-    auto issue_pv = [&](int st, int n, uint32_t first) {
-      const uint32_t vb = kv_base + ((2 * n + 1) % NSTAGE) * L::KV_BYTES;
+    // Descriptors: the high word is fixed (SBO 1024, version 1, 128B swizzle); the low
+    // word is (address >> 4) | LBO << 16, so stepping through a tile is one add.
+    constexpr uint32_t DESC_HI = (1024u >> 4) | (1u << 14) | (2u << 29);
+    constexpr uint32_t LBO_K = 1u << 16;                                           // K-major: LBO unused
+    constexpr uint32_t LBO_V = (uint32_t)(L::HALF_BYTES >> 4) << 16;              // MN-major: next 64 dims
+    auto desc = [&](uint32_t lo) { return (static_cast<uint64_t>(DESC_HI) << 32) | lo; };
+    const uint32_t kv_lo = kv_base >> 4, q_lo = (q_base >> 4) | LBO_K;
+    // O_st (+)= P_st V for half h (keys 64h..64h+63) of KV tile n (ring load 2n+1); P from TMEM
+    auto issue_pv_half = [&](int st, int n, int h, uint32_t first) {
+      const uint32_t v_lo = (kv_lo + ((2 * n + 1) % NSTAGE) * (L::KV_BYTES >> 4)) | LBO_V;
 #pragma unroll
-      for (int k = 0; k < BN / 16; ++k) {
-        const uint64_t b = smem_desc(vb + k * 2048, L::HALF_BYTES, 1024);     // MN-major: LBO = next 64 dims
-        umma_bf16_ts(tmem_O + st * D, tmem_S + st * BN + k * 8, b, IDESC_PV, (!first || k > 0) ? 1u : 0u);
-      }
+      for (int k = 4 * h; k < 4 * h + 4; ++k)
+        umma_bf16_ts(tmem_O + st * D, tmem_S + st * BN + k * 8, desc(v_lo + k * (2048 >> 4)), IDESC_PV,
+                     (!first || k > 0) ? 1u : 0u);
     };
     auto issue_qk = [&](int st, int n) {
-      const uint32_t kb = kv_base + ((2 * n) % NSTAGE) * L::KV_BYTES;
-      const uint32_t qb = q_base + (dual ? st : 0) * L::Q_BYTES;
+      const uint32_t k_lo = (kv_lo + ((2 * n) % NSTAGE) * (L::KV_BYTES >> 4)) | LBO_K;
+      const uint32_t a_lo = q_lo + (dual ? st : 0) * (L::Q_BYTES >> 4);
 #pragma unroll
       for (int k = 0; k < D / 16; ++k) {
-        const uint32_t off = (k >> 2) * L::HALF_BYTES + (k & 3) * 32;
-        umma_bf16(tmem_S + st * BN, smem_desc(qb + off, 16, 1024), smem_desc(kb + off, 16, 1024), IDESC_QK,
-                  k > 0 ? 1u : 0u);
+        const uint32_t off = ((k >> 2) * L::HALF_BYTES + (k & 3) * 32) >> 4;
+        umma_bf16(tmem_S + st * BN, desc(a_lo + off), desc(k_lo + off), IDESC_QK, k > 0 ? 1u : 0u);
       }
     };
     // V rows past the visible range hold stale or foreign data; P is 0 there but
@@ -485,24 +503,30 @@ prefill_tc_kernel(const Params p, const __grid_constant__ CUtensorMap map_k, con
         const int my_cnt = st == 0 ? cnt0 : cnt1;
         if (my_cnt == 0 || k > my_cnt) continue;
         const bool last_user = !dual || st == 1;            // last stream to touch this K/V tile
-        if (k > 0) {
+        if (k > 0 && pv_role) {
           const int n = dual ? k - 1 : 2 * (k - 1) + st;
           const int lv = 2 * n + 1;
           mbar_wait(bar(BAR_FULL + lv % NSTAGE), (lv / NSTAGE) & 1, abort_flag, p.status);
           if (!dual || st == 0) clear_v_tail(n);
-          mbar_wait(bar(BAR_P + st), (k - 1) & 1, abort_flag, p.status);
-          tc_fence_after();
+#pragma unroll
+          for (int h = 0; h < 2; ++h) {
+            mbar_wait(bar(BAR_P + 2 * st + h), (k - 1) & 1, abort_flag, p.status);
+            tc_fence_after();
+            if (lane == 0) issue_pv_half(st, n, h, k == 1);
+          }
           if (lane == 0) {
-            issue_pv(st, n, k == 1);
             if (last_user) tc_commit(bar(BAR_EMPTY + lv % NSTAGE));
             if (k == my_cnt) tc_commit(bar(BAR_O + st));
+            tc_fence_before();
+            mbar_arrive(bar(BAR_PVI + st));                   // PV(k-1) is issued: S/P columns may be rewritten
           }
           __syncwarp();
         }
-        if (k < my_cnt) {
+        if (k < my_cnt && !pv_role) {
           const int n = dual ? k : 2 * k + st;
           const int lk = 2 * n;
           mbar_wait(bar(BAR_FULL + lk % NSTAGE), (lk / NSTAGE) & 1, abort_flag, p.status);
+          if (k > 0) mbar_wait(bar(BAR_PVI + st), (k - 1) & 1, abort_flag, p.status);
           tc_fence_after();
           if (lane == 0) {
             issue_qk(st, n);
@@ -615,10 +639,21 @@ Plan make_plan(const efim_cache_desc* c, const efim_batch_desc* b, WorkItem* ite
     }
   }
   if (items) {
-    // longest first, so the tail of the launch is made of short items
-    std::stable_sort(items, items + n_items, [](const WorkItem& a, const WorkItem& b2) {
-      return (a.tile_end - a.tile_begin) > (b2.tile_end - b2.tile_begin);
-    });
+    if (n_items > 8 * 148) {
+      // Many waves: CTAs that run together should read the same K/V.  Keep the row tiles
+      // of one (sequence, kv head) adjacent (longest first inside the group), so the
+      // concurrent working set is a few heads' K/V and stays in L2.
+      std::stable_sort(items, items + n_items, [](const WorkItem& a, const WorkItem& b2) {
+        if (a.seq != b2.seq) return a.seq < b2.seq;
+        if (a.kvh != b2.kvh) return a.kvh < b2.kvh;
+        return a.row0 > b2.row0;
+      });
+    } else {
+      // Few waves: longest first, so the tail of the launch is made of short items
+      std::stable_sort(items, items + n_items, [](const WorkItem& a, const WorkItem& b2) {
+        return (a.tile_end - a.tile_begin) > (b2.tile_end - b2.tile_begin);
+      });
+    }
   }
   pl.n_items = (int)n_items;
   pl.s_max = s_max;
