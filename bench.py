@@ -46,6 +46,24 @@ def load_peaks():
     return p
 
 
+def recorded_traffic(workload, call):
+    """DRAM bytes per launch of `call` on `workload` from the committed ncu summary, or
+    None when there is none or the kernel source changed since it was taken."""
+    import glob
+    import hashlib
+    for path in glob.glob(os.path.join(ROOT, "profiles", "dram_traffic_*.txt")):
+        for line in open(path):
+            if not line.startswith("traffic "):
+                continue
+            kv = dict(tok.split("=", 1) for tok in line.split()[1:])
+            if kv.get("workload") != workload or kv.get("call") != call:
+                continue
+            src = os.path.join(ROOT, kv["source"])
+            if os.path.exists(src) and hashlib.sha1(open(src, "rb").read()).hexdigest() == kv["sha1"]:
+                return int(kv["dram_bytes"])
+    return None
+
+
 def workload_counts(w):
     """Algorithmic work of one step (unmasked pairs, each K/V byte once)."""
     C = w.cached_len.astype(np.int64)
@@ -390,7 +408,10 @@ def run_native(args):
                 "peak": peaks["hbm_gbs"], "unit": "GB/s"}
     roof["frac"] = roof["achieved"] / roof["peak"]
     roof["peak_source"] = peaks["source"]
-    roof["traffic"] = None
+    roof["traffic"] = recorded_traffic(w.name if args.batch is None else None, roof["kernel"])
+    roof["traffic_unit"] = "bytes/launch (ncu dram read+write)"
+    roof["algorithmic"] = cnt["prefill_kv_bytes"] if roof["kernel"] == "efim_append_prefill_attn" and roof["bound"] == "hbm" \
+        else (cnt["prefill_flops"] if roof["kernel"] == "efim_append_prefill_attn" else cnt["decode_kv_bytes"])
     roof["intensity_flop_per_byte"] = intensity
 
     # ---------------- CPU oracle on a bounded sample (rank 0, N = 1 only)
