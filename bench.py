@@ -178,7 +178,7 @@ def oracle_threads():
         return os.cpu_count() or 1
 
 
-def pick_sample(w, budget_flops=1.2e11):
+def pick_sample(w, budget_flops=3.6e11):
     """Sequences of the workload, shortest first, until ~budget of oracle work."""
     C = w.cached_len.astype(np.int64)
     N = w.new_len.astype(np.int64)
@@ -454,7 +454,7 @@ def run_native(args):
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=20)
+    ap.add_argument("--steps", type=int, default=100)
     ap.add_argument("--warmup", type=int, default=5)
     ap.add_argument("--impl", default="native", choices=["native", "reference"])
     ap.add_argument("--workload", default="cfg2")
