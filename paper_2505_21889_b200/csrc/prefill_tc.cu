@@ -290,7 +290,9 @@ prefill_tc_kernel(const Params p, const __grid_constant__ CUtensorMap map_k, con
       const float mx = fmaxf(fmaxf(fmaxf(mx8[0], mx8[1]), fmaxf(mx8[2], mx8[3])),
                              fmaxf(fmaxf(mx8[4], mx8[5]), fmaxf(mx8[6], mx8[7])));
       const float m_new = mx * p.scale_log2;
-      // lazy rescale: keep the old reference maximum until it is off by more than 2^8
+      // lazy rescale: keep the old reference maximum until it is off by more than 2^8.
+      // O is quiet here: QK(k) was issued after PV(k-1) (barrier PVI) and the tensor pipe
+      // completes in order, so S(k) being ready means PV(k-1) has landed.
       const bool grow = m_new > m_ref + 8.f;
       if (k == 0) {
         m_ref = m_new;
