@@ -84,7 +84,11 @@ __global__ void __launch_bounds__(128) decode_splitkv_kernel(const DecodeParams 
   const int g0 = (blockIdx.y % gsplit) * GT;
   const int ng = min(GT, G - g0);
   const int c = blockIdx.z;
-  const int len = __ldg(p.row_len + r);
+  int len = __ldg(p.row_len + r);
+  if (len > p.max_pages_per_seq * 16) {           // longer than the block table can address: clamp and report
+    len = p.max_pages_per_seq * 16;
+    if (threadIdx.x == 0 && p.status) atomicOr(p.status, EFIM_DEV_BAD_POSITION);
+  }
   const int begin = c * p.chunk_tokens;
   const int head0 = kvh * G + g0;
   const int tid = threadIdx.x;
@@ -349,7 +353,7 @@ __global__ void __launch_bounds__(128) decode_merge_kernel(const DecodeParams p)
   const size_t row_head = (size_t)blockIdx.x * 4 + (threadIdx.x >> 5);
   if (row_head >= (size_t)p.R * p.Hq) return;
   const int r = (int)(row_head / p.Hq);
-  const int len = __ldg(p.row_len + r);
+  const int len = min(__ldg(p.row_len + r), p.max_pages_per_seq * 16);
   uint16_t* out = p.out + row_head * D + lane * EPL;
   if (len <= 0) {
 #pragma unroll

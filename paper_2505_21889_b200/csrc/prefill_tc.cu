@@ -418,7 +418,8 @@ prefill_tc_kernel(const Params p, const __grid_constant__ CUtensorMap map_k, con
       const int keys = min(BN, kv_cap - tile * BN);
       const int npages = keys > 0 ? (keys + 15) >> 4 : 0;
       int pid = -1;
-      const bool want = page_l < npages && lane < 8 * HALVES;
+      // (the second test only matters if the device lengths disagree with the host mirrors)
+      const bool want = page_l < npages && lane < 8 * HALVES && tile * 8 + page_l < p.max_pages_per_seq;
       if (want) pid = __ldg(bt + tile * 8 + page_l);
       const bool ok = want && pid >= 0 && pid < p.num_pages;
       if (want && !ok && p.status) atomicOr(p.status, EFIM_DEV_BAD_PAGE);

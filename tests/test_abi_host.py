@@ -91,3 +91,47 @@ def test_bad_arguments_are_rejected_on_the_host():
     # empty batch is a no-op
     bd0 = B._BatchDesc(0, 4, 0, None, None, None, None, None, None)
     assert lib.efim_kv_append(ctypes.byref(ok), ctypes.byref(bd0), None, None, None, None, None, None) == 0
+
+
+def _batch_desc(cached, new, max_pages):
+    c = np.asarray(cached, np.int32)
+    n = np.asarray(new, np.int32)
+    bd = B._BatchDesc(len(c), max_pages, int(n.sum()), 0x1000, 0x1000, 0x1000, 0x1000, c.ctypes.data, n.ctypes.data)
+    bd._keep = (c, n)
+    return bd
+
+
+def test_prefill_planner_splits_few_long_items_and_not_many_short_ones():
+    """Host planning of efim_append_prefill_attn, seen through its two queries: few long
+    work items get their key range split (partials + a merge launch), many items do not."""
+    lib = efim.load_library()
+    cache = _cache_desc(Hq=32, Hkv=8)
+    # cfg4a-like: 8 sequences x 8 kv heads x 2 row tiles = 128 items of 65 key tiles -> split
+    few = _batch_desc([8192] * 8, [128] * 8, 600)
+    assert lib.efim_prefill_launch_count(ctypes.byref(cache), ctypes.byref(few)) == 2
+    ws_few = lib.efim_prefill_workspace_bytes(ctypes.byref(cache), ctypes.byref(few))
+    rows = 8 * 128 * 32
+    assert ws_few > rows * 128 * 4 * 2            # room for at least two fp32 partials per (token, head)
+    # cfg4b-like: 3200 items -> one launch, workspace is just the work list
+    many = _batch_desc([5120] * 8, [3200] * 8, 600)
+    assert lib.efim_prefill_launch_count(ctypes.byref(cache), ctypes.byref(many)) == 1
+    ws_many = lib.efim_prefill_workspace_bytes(ctypes.byref(cache), ctypes.byref(many))
+    items = 8 * 8 * (3200 * 4 // 256)
+    assert items * 32 <= ws_many < items * 32 + 4096
+    # nothing new -> nothing to do
+    none = _batch_desc([100, 200], [0, 0], 32)
+    assert lib.efim_prefill_launch_count(ctypes.byref(cache), ctypes.byref(none)) == 0
+    assert lib.efim_prefill_workspace_bytes(ctypes.byref(cache), ctypes.byref(none)) == 0
+
+
+def test_decode_planner_chunks():
+    lib = efim.load_library()
+    cache = _cache_desc(Hq=32, Hkv=8)
+    # large batch x long context: chunks of 2048 keys, merge needed
+    assert lib.efim_decode_launch_count(ctypes.byref(cache), 256, 32832) == 2
+    ws = lib.efim_decode_workspace_bytes(ctypes.byref(cache), 256, 32832)
+    n_chunks = -(-32832 // 2048)
+    assert ws >= 256 * 32 * n_chunks * 129 * 4
+    # a context of one chunk needs neither workspace nor merge
+    assert lib.efim_decode_launch_count(ctypes.byref(cache), 4096, 200) == 1
+    assert lib.efim_decode_workspace_bytes(ctypes.byref(cache), 4096, 200) == 0
