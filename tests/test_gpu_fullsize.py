@@ -70,7 +70,8 @@ def test_cfg5_full_decode_steps_sampled():
     seqs = sorted([int(order[0]), int(order[-1]), int(order[100])])
     kp, vp, bt, seqs = w.compact_host_pool(seqs)
     B = w.batch
-    steps = 3
+    steps = w.decode_steps                       # all 64; the oracle checks steps 0, 31 and 63
+    check = {0, 31, steps - 1}
     max_ctx = int(ctx_all.max()) + w.decode_steps
     ws = torch.empty(max(efim.efim_decode_workspace_bytes(dw.cache, B, max_ctx), 256), dtype=torch.uint8, device="cuda")
     one_all = np.ones(B, np.int32)
@@ -82,15 +83,17 @@ def test_cfg5_full_decode_steps_sampled():
         sb = efim.Batch(ctx_all, one_all, dw.batch.d_block_table)
         ctx_all = ctx_all + 1
         ctx = ctx + 1
-        o, lse = orc.decode_attention(q_rot, kp, vp, bt, ctx, w.num_q_heads)
         dq, dk, dv = H.bits_to_torch(q), H.bits_to_torch(k), H.bits_to_torch(v)
         efim.efim_kv_append(dw.cache, sb, dw.rope, dq, dk, dv, dw.status)
         out = torch.empty_like(dq)
         lse_d = torch.empty((B, w.num_q_heads), dtype=torch.float32, device="cuda")
         efim.efim_decode_attn(dw.cache, B, torch.from_numpy(ctx_all).cuda(), max_ctx, dw.batch.d_block_table, dq, out,
                               lse_d, 0.0, ws, dw.status)
+        if step not in check:
+            continue
         torch.cuda.synchronize()
         assert int(dw.status.item()) == 0
+        o, lse = orc.decode_attention(q_rot, kp, vp, bt, ctx, w.num_q_heads)
         H.assert_attn_close(H.torch_to_bits(out)[seqs], o, f"cfg5 full decode step {step}")
         assert np.abs(lse_d.cpu().numpy()[seqs] - lse).max() <= H.LSE_TOL
         assert torch.isfinite(out.float()).all()

@@ -181,6 +181,13 @@ def test_decode_zero_length_and_bad_page_flag():
     torch.cuda.synchronize()
     assert int(dw.status.item()) & 0x1
     assert torch.isfinite(out.float()).all()
+    # a device length beyond what the block table addresses is clamped and reported
+    dw.status.zero_()
+    cap = dw.batch.d_block_table.shape[1] * 16
+    too_long = torch.tensor([40, 0, cap + 100], dtype=torch.int32, device="cuda")
+    efim.efim_decode_attn(dw.cache, 3, too_long, 96, dw.batch.d_block_table, q, out, lse, 0.0, ws, dw.status)
+    torch.cuda.synchronize()
+    assert int(dw.status.item()) & 0x2
 
 
 def test_pages_outside_the_batch_are_untouched():
