@@ -5,8 +5,8 @@
 // One CTA owns up to 256 packed query rows (row = token * G + head-in-group) of one
 // (sequence, kv head) as two 128-row tiles, and streams the visible K/V range in
 // tiles of 128 keys (8 pages):
-//   warp 8    TMA producer: walks the block table, one tiled bulk-tensor copy per
-//             (page, 64-dim half) into a 5-entry shared-memory ring (128B swizzle)
+//   warps 8,11 TMA producers (K tiles / V tiles): walk the block table, one tiled bulk-tensor
+//             copy per (page, 64-dim half) into a 5- or 6-entry shared-memory ring (128B swizzle)
 //   warp 10   issues the tcgen05.mma for S_t = Q_t K^T into TMEM
 //   warp 9    issues the tcgen05.mma for O_t += P_t V (P read from TMEM)
 //   warps 0-7 two softmax groups, one per query tile, one TMEM lane (row) per thread:
@@ -161,8 +161,8 @@ struct Smem {
 // barrier slots (8 bytes each) inside the BAR_OFF block
 // (P has two barriers per stream: keys 0-63 and 64-127 of a tile are handed over separately)
 enum {
-  BAR_Q = 0, BAR_S = 2, BAR_P = 4, BAR_O = 8, BAR_PVI = 10, BAR_FULL = 12, BAR_EMPTY = 12 + NSTAGE,
-  BAR_COUNT = 12 + 2 * NSTAGE
+  BAR_Q = 0, BAR_S = 2, BAR_P = 4, BAR_O = 8, BAR_PVI = 10, BAR_FULL = 12, BAR_EMPTY = 12 + NSTAGE_MAX,
+  BAR_COUNT = 12 + 2 * NSTAGE_MAX
 };
 
 // Two softmax groups ("streams") run per CTA.  With more than 128 rows, stream t
@@ -170,9 +170,9 @@ enum {
 // one query tile; stream 0 takes the even KV tiles and stream 1 the odd ones, each
 // with its own running (max, sum, O), and the two states are merged at the end -
 // the tensor core then still works on one stream while the other does its softmax.
-template <int D>
-__global__ void __launch_bounds__(THREADS, 1)
-prefill_tc_kernel(const Params p, const __grid_constant__ CUtensorMap map_k, const __grid_constant__ CUtensorMap map_v) {
+template <int D, bool DUAL>
+__device__ __forceinline__ void prefill_tc_body(const Params& p, const CUtensorMap& map_k, const CUtensorMap& map_v,
+                                                const WorkItem& it) {
   using L = Smem<D>;
   constexpr int HALVES = L::HALVES;
   extern __shared__ uint8_t smem_raw[];
@@ -184,19 +184,26 @@ prefill_tc_kernel(const Params p, const __grid_constant__ CUtensorMap map_k, con
   auto bar = [&](int i) { return bars + 8u * i; };
 
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
-  const WorkItem it = p.items[blockIdx.x];
   const int G = p.G;
   const int C = __ldg(p.cached_len + it.seq);
   const int N = __ldg(p.new_len + it.seq);
   const int tok0 = __ldg(p.q_indptr + it.seq);
   const int rows_total = N * G;
   const int rows_here = min(NQ * BM, rows_total - it.row0);
-  const bool dual = rows_here > BM;                          // two query tiles
+  constexpr bool dual = DUAL;                                // two query tiles (rows_here > BM)
   const int i_last = (it.row0 + rows_here - 1) / G;          // last token of this CTA
   const int kv_cap = C + i_last + 1;                         // keys any row here may see
   const int nt = it.tile_end - it.tile_begin;
   const int cnt0 = dual ? nt : (nt + 1) >> 1;                // KV tiles of stream 0 / 1
   const int cnt1 = dual ? nt : nt >> 1;
+  // K/V ring.  With one query tile the second tile's shared memory joins the ring
+  // (6 entries instead of 5), and the loads are ordered the way the two streams consume
+  // them - K0 K1 V0 K2 V1 K3 ... - so that no entry sits loaded but unused for a whole
+  // period: such CTAs stream their K/V alone and live on the bytes they keep in flight.
+  constexpr int nst = dual ? NSTAGE : NSTAGE_MAX;
+  constexpr uint32_t ring_off = dual ? L::KV_OFF : L::KV_OFF - L::KV_BYTES;
+  auto ld_k = [&](int n) { return dual ? 2 * n : (n == 0 ? 0 : 2 * n - 1); };          // ring load index of K(n)
+  auto ld_v = [&](int n) { return dual ? 2 * n + 1 : min(2 * n + 2, 2 * nt - 1); };    // ... of V(n)
 
   if (tid == 0) {
     for (int t = 0; t < NQ; ++t) {
@@ -207,7 +214,7 @@ prefill_tc_kernel(const Params p, const __grid_constant__ CUtensorMap map_k, con
       mbar_init(bar(BAR_O + t), 1);
       mbar_init(bar(BAR_PVI + t), 1);
     }
-    for (int s = 0; s < NSTAGE; ++s) {
+    for (int s = 0; s < NSTAGE_MAX; ++s) {
       mbar_init(bar(BAR_FULL + s), 1);
       mbar_init(bar(BAR_EMPTY + s), 1);
     }
@@ -409,39 +416,50 @@ prefill_tc_kernel(const Params p, const __grid_constant__ CUtensorMap map_k, con
       }
     }
     tc_fence_before();
-  } else if (warp == 8) {
-    // ============================================================ TMA producer
+  } else if (warp == 8 || warp == 11) {
+    // ============================================================ TMA producers
+    // Every bulk-tensor copy costs its issuing warp ~65 cycles and a 128-key tile takes
+    // 16 of them (one 2 KB box per page and 64-dim half), so one warp tops out near
+    // 30 GB/s.  Warp 8 therefore loads the K tiles and warp 11 the V tiles.
+    const int my_which = warp == 8 ? 0 : 1;
     const int32_t* bt = p.block_table + (size_t)it.seq * p.max_pages_per_seq;
     const int page_l = lane / HALVES, half_l = lane % HALVES;
-    for (int jj = 0; jj < nt; ++jj) {
+    const CUtensorMap* my_map = my_which == 0 ? &map_k : &map_v;
+    // this lane's page id for tile jj, or -1 (lanes beyond the tile's pages, table overrun)
+    auto lookup = [&](int jj) {
+      if (jj >= nt) return -1;
       const int tile = it.tile_begin + jj;
       const int keys = min(BN, kv_cap - tile * BN);
       const int npages = keys > 0 ? (keys + 15) >> 4 : 0;
-      int pid = -1;
-      // (the second test only matters if the device lengths disagree with the host mirrors)
+      // (the last test only matters if the device lengths disagree with the host mirrors)
       const bool want = page_l < npages && lane < 8 * HALVES && tile * 8 + page_l < p.max_pages_per_seq;
-      if (want) pid = __ldg(bt + tile * 8 + page_l);
-      const bool ok = want && pid >= 0 && pid < p.num_pages;
-      if (want && !ok && p.status) atomicOr(p.status, EFIM_DEV_BAD_PAGE);
+      return want ? __ldg(bt + tile * 8 + page_l) : -1;
+    };
+    // the block-table read is a dependent global load in front of every copy: fetch it two tiles ahead
+    int pid_a = lookup(0), pid_b = lookup(1);
+    for (int jj = 0; jj < nt; ++jj) {
+      const int pid = pid_a;
+      pid_a = pid_b;
+      pid_b = lookup(jj + 2);
+      const int ld = my_which == 0 ? ld_k(jj) : ld_v(jj);
+      const bool ok = pid >= 0 && pid < p.num_pages;
+      if (pid >= p.num_pages && my_which == 0 && p.status) atomicOr(p.status, EFIM_DEV_BAD_PAGE);
       const uint32_t okmask = __ballot_sync(0xffffffffu, ok);
       const uint32_t bytes = __popc(okmask) * 2048u;
-#pragma unroll
-      for (int which = 0; which < 2; ++which) {
-        const int ld = 2 * jj + which;
-        const int slot = ld % NSTAGE, use = ld / NSTAGE;
-        mbar_wait(bar(BAR_EMPTY + slot), (use & 1) ^ 1, abort_flag, p.status);
-        if (lane == 0) mbar_expect_tx(bar(BAR_FULL + slot), bytes);
-        __syncwarp();
-        if (ok) {
-          const uint32_t dst = smem_base + L::KV_OFF + slot * L::KV_BYTES + half_l * L::HALF_BYTES + page_l * 2048;
-          tma_load_4d(dst, which == 0 ? &map_k : &map_v, bar(BAR_FULL + slot), half_l * 64, 0, it.kvh, pid);
-        }
+      const int slot = ld % nst, use = ld / nst;
+      mbar_wait(bar(BAR_EMPTY + slot), (use & 1) ^ 1, abort_flag, p.status);
+      if (lane == 0) mbar_expect_tx(bar(BAR_FULL + slot), bytes);
+      __syncwarp();
+      if (ok) {
+        const uint32_t dst = smem_base + ring_off + slot * L::KV_BYTES + half_l * L::HALF_BYTES + page_l * 2048;
+        tma_load_4d(dst, my_map, bar(BAR_FULL + slot), half_l * 64, 0, it.kvh, pid);
       }
     }
     // if the CTA gave up, let copies that are still in flight land before shared memory goes away
     if (*abort_flag) {
-      for (int ld = max(0, 2 * nt - NSTAGE); ld < 2 * nt; ++ld) {
-        const uint32_t b = bar(BAR_FULL + ld % NSTAGE), par = (ld / NSTAGE) & 1;
+      for (int jj = max(0, nt - nst); jj < nt; ++jj) {
+        const int ld = my_which == 0 ? ld_k(jj) : ld_v(jj);
+        const uint32_t b = bar(BAR_FULL + ld % nst), par = (ld / nst) & 1;
         for (int spin = 0; spin < (1 << 20) && !mbar_try(b, par); ++spin) {}
       }
     }
@@ -455,7 +473,7 @@ prefill_tc_kernel(const Params p, const __grid_constant__ CUtensorMap map_k, con
     const bool pv_role = warp == 9;
     constexpr uint32_t IDESC_QK = instr_desc(BN, 0);
     constexpr uint32_t IDESC_PV = instr_desc(D, 1);
-    const uint32_t q_base = smem_base + L::Q_OFF, kv_base = smem_base + L::KV_OFF;
+    const uint32_t q_base = smem_base + L::Q_OFF, kv_base = smem_base + ring_off;
     mbar_wait(bar(BAR_Q + 0), 0, abort_flag, p.status);
     if (dual) mbar_wait(bar(BAR_Q + 1), 0, abort_flag, p.status);
     tc_fence_after();
@@ -468,14 +486,14 @@ prefill_tc_kernel(const Params p, const __grid_constant__ CUtensorMap map_k, con
     const uint32_t kv_lo = kv_base >> 4, q_lo = (q_base >> 4) | LBO_K;
     // O_st (+)= P_st V for half h (keys 64h..64h+63) of KV tile n (ring load 2n+1); P from TMEM
     auto issue_pv_half = [&](int st, int n, int h, uint32_t first) {
-      const uint32_t v_lo = (kv_lo + ((2 * n + 1) % NSTAGE) * (L::KV_BYTES >> 4)) | LBO_V;
+      const uint32_t v_lo = (kv_lo + (ld_v(n) % nst) * (L::KV_BYTES >> 4)) | LBO_V;
 #pragma unroll
       for (int k = 4 * h; k < 4 * h + 4; ++k)
         umma_bf16_ts(tmem_O + st * D, tmem_S + st * BN + k * 8, desc(v_lo + k * (2048 >> 4)), IDESC_PV,
                      (!first || k > 0) ? 1u : 0u);
     };
     auto issue_qk = [&](int st, int n) {
-      const uint32_t k_lo = (kv_lo + ((2 * n) % NSTAGE) * (L::KV_BYTES >> 4)) | LBO_K;
+      const uint32_t k_lo = (kv_lo + (ld_k(n) % nst) * (L::KV_BYTES >> 4)) | LBO_K;
       const uint32_t a_lo = q_lo + (dual ? st : 0) * (L::Q_BYTES >> 4);
 #pragma unroll
       for (int k = 0; k < D / 16; ++k) {
@@ -488,7 +506,7 @@ prefill_tc_kernel(const Params p, const __grid_constant__ CUtensorMap map_k, con
     auto clear_v_tail = [&](int n) {
       const int keys = kv_cap - (it.tile_begin + n) * BN;
       if (keys < BN) {
-        uint8_t* vb = smem_gen + L::KV_OFF + ((2 * n + 1) % NSTAGE) * L::KV_BYTES;
+        uint8_t* vb = smem_gen + ring_off + (ld_v(n) % nst) * L::KV_BYTES;
         const int first = max(keys, 0);
         const int chunks = (BN - first) * 8 * HALVES;       // 16-byte chunks to clear
         for (int idx = lane; idx < chunks; idx += 32) {
@@ -508,8 +526,8 @@ prefill_tc_kernel(const Params p, const __grid_constant__ CUtensorMap map_k, con
         const bool last_user = !dual || st == 1;            // last stream to touch this K/V tile
         if (k > 0 && pv_role) {
           const int n = dual ? k - 1 : 2 * (k - 1) + st;
-          const int lv = 2 * n + 1;
-          mbar_wait(bar(BAR_FULL + lv % NSTAGE), (lv / NSTAGE) & 1, abort_flag, p.status);
+          const int lv = ld_v(n);
+          mbar_wait(bar(BAR_FULL + lv % nst), (lv / nst) & 1, abort_flag, p.status);
           if (!dual || st == 0) clear_v_tail(n);
 #pragma unroll
           for (int h = 0; h < 2; ++h) {
@@ -518,7 +536,7 @@ prefill_tc_kernel(const Params p, const __grid_constant__ CUtensorMap map_k, con
             if (lane == 0) issue_pv_half(st, n, h, k == 1);
           }
           if (lane == 0) {
-            if (last_user) tc_commit(bar(BAR_EMPTY + lv % NSTAGE));
+            if (last_user) tc_commit(bar(BAR_EMPTY + lv % nst));
             if (k == my_cnt) tc_commit(bar(BAR_O + st));
             tc_fence_before();
             mbar_arrive(bar(BAR_PVI + st));                   // PV(k-1) is issued: S/P columns may be rewritten
@@ -527,14 +545,14 @@ prefill_tc_kernel(const Params p, const __grid_constant__ CUtensorMap map_k, con
         }
         if (k < my_cnt && !pv_role) {
           const int n = dual ? k : 2 * k + st;
-          const int lk = 2 * n;
-          mbar_wait(bar(BAR_FULL + lk % NSTAGE), (lk / NSTAGE) & 1, abort_flag, p.status);
+          const int lk = ld_k(n);
+          mbar_wait(bar(BAR_FULL + lk % nst), (lk / nst) & 1, abort_flag, p.status);
           if (k > 0) mbar_wait(bar(BAR_PVI + st), (k - 1) & 1, abort_flag, p.status);
           tc_fence_after();
           if (lane == 0) {
             issue_qk(st, n);
             tc_commit(bar(BAR_S + st));
-            if (last_user) tc_commit(bar(BAR_EMPTY + lk % NSTAGE));
+            if (last_user) tc_commit(bar(BAR_EMPTY + lk % nst));
           }
           __syncwarp();
         }
@@ -547,6 +565,19 @@ prefill_tc_kernel(const Params p, const __grid_constant__ CUtensorMap map_k, con
     tc_fence_after();
     asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem), "r"(512u) : "memory");
   }
+}
+
+template <int D>
+__global__ void __launch_bounds__(THREADS, 1)
+prefill_tc_kernel(const Params p, const __grid_constant__ CUtensorMap map_k, const __grid_constant__ CUtensorMap map_v) {
+  const WorkItem it = p.items[blockIdx.x];
+  const int rows_here = __ldg(p.new_len + it.seq) * p.G - it.row0;
+  // the two shapes of a CTA are separate instantiations: ring size, load order and the
+  // query-tile choice are compile-time constants in the issuing warps' inner loops
+  if (rows_here > BM)
+    prefill_tc_body<D, true>(p, map_k, map_v, it);
+  else
+    prefill_tc_body<D, false>(p, map_k, map_v, it);
 }
 
 // Merge the KV-chunk partials of split sequences: one warp per (token, head).

@@ -10,7 +10,8 @@ constexpr int BM = 128;        // query rows per tile (one TMEM lane each)
 constexpr int BN = 128;        // keys per KV tile (8 pages)
 constexpr int NQ = 2;          // query tiles per CTA sharing one K/V stream
 constexpr int NSTAGE = 5;      // K/V ring entries (one K or V tile of 128 keys each)
-constexpr int THREADS = 384;   // 2 softmax warpgroups + 1 service warpgroup (TMA warp, MMA warp, 2 spare)
+constexpr int NSTAGE_MAX = 6;  // ring entries when there is a single query tile (the other tile's space is used)
+constexpr int THREADS = 384;   // 2 softmax warpgroups + 1 service warpgroup (2 TMA warps, 2 MMA warps)
 // Register split (setmaxnreg): the block launches with 168 registers per thread
 // (65536 / 384, rounded to 8) = 64512 in total; 2 x 128 x 216 + 128 x 64 = 63488 fits.
 constexpr int REGS_SOFTMAX = 216;
