@@ -60,6 +60,8 @@ typedef enum {
 #define EFIM_DEV_TIMEOUT       0x4   /* a bounded wait inside a kernel expired               */
 
 const char* efim_strerror(efim_status s);
+/* Text of the CUDA error behind the calling thread's most recent EFIM_ERR_CUDA. */
+const char* efim_last_cuda_error(void);
 int efim_version(void);
 
 /* Paged KV cache of ONE layer. */

@@ -14,7 +14,8 @@ _HERE = os.path.dirname(os.path.abspath(__file__))
 class EfimError(RuntimeError):
     def __init__(self, code, where):
         self.code = int(code)
-        super().__init__(f"{where}: {efim_strerror(code)} (status {int(code)})")
+        detail = f" [{load_library().efim_last_cuda_error().decode()}]" if int(code) == 5 else ""
+        super().__init__(f"{where}: {efim_strerror(code)} (status {int(code)}){detail}")
 
 
 class _CacheDesc(Structure):
@@ -33,7 +34,7 @@ class _RopeDesc(Structure):
     _fields_ = [("d_cos_sin", c_void_p), ("max_position", c_int32), ("interleaved", c_int32)]
 
 
-EXPORTS = ("efim_strerror", "efim_version", "efim_rope_table_build", "efim_kv_append",
+EXPORTS = ("efim_last_cuda_error", "efim_strerror", "efim_version", "efim_rope_table_build", "efim_kv_append",
            "efim_prefill_workspace_bytes", "efim_append_prefill_attn",
            "efim_decode_workspace_bytes", "efim_decode_attn",
            "efim_decode_static_scratch_bytes", "efim_decode_attn_static",
@@ -56,6 +57,7 @@ def load_library():
     lib = ctypes.CDLL(path)
     lib.efim_strerror.restype = c_char_p
     lib.efim_strerror.argtypes = [ctypes.c_int]
+    lib.efim_last_cuda_error.restype = c_char_p
     lib.efim_version.restype = ctypes.c_int
     lib.efim_rope_table_build.restype = ctypes.c_int
     lib.efim_rope_table_build.argtypes = [c_double, c_int32, c_int32, c_void_p]

@@ -1,5 +1,14 @@
 // Status strings and version of the EFIM C ABI.
+#include <cuda_runtime.h>
 #include "efim.h"
+
+static thread_local int g_last_cuda_error = 0;
+
+extern "C" void efim_note_cuda_error(int code) { g_last_cuda_error = code; }
+
+extern "C" const char* efim_last_cuda_error(void) {
+  return g_last_cuda_error ? cudaGetErrorString(static_cast<cudaError_t>(g_last_cuda_error)) : "no error";
+}
 
 extern "C" const char* efim_strerror(efim_status s) {
   switch (s) {

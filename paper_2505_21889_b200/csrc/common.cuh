@@ -5,10 +5,16 @@
 #include <stdint.h>
 #include "efim.h"
 
+// the CUDA error behind the calling thread's last EFIM_ERR_CUDA (api.cu)
+extern "C" void efim_note_cuda_error(int code);
+
 #define EFIM_CUDA_TRY(expr)                          \
   do {                                               \
     cudaError_t e__ = (expr);                        \
-    if (e__ != cudaSuccess) return EFIM_ERR_CUDA;    \
+    if (e__ != cudaSuccess) {                        \
+      efim_note_cuda_error((int)e__);                \
+      return EFIM_ERR_CUDA;                          \
+    }                                                \
   } while (0)
 
 namespace efim {

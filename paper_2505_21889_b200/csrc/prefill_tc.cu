@@ -561,6 +561,12 @@ __device__ __forceinline__ void prefill_tc_body(const Params& p, const CUtensorM
     tc_fence_before();
   }
   __syncthreads();
+  if (*abort_flag) {
+    // a wait expired: roles ran out of step, copies and MMAs may still be in flight; give
+    // them a generous moment to finish before TMEM and shared memory are released
+    for (int i = 0; i < 2000; ++i) __nanosleep(1000);
+    __syncthreads();
+  }
   if (warp == 9) {
     tc_fence_after();
     asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem), "r"(512u) : "memory");
