@@ -17,6 +17,7 @@
 #include "prefill_tc.cuh"
 #include <vector>
 #include <algorithm>
+#include <functional>
 
 namespace efim {
 namespace pf {
@@ -253,7 +254,9 @@ __device__ __forceinline__ void prefill_tc_body(const Params& p, const CUtensorM
     const bool valid = R < rows_total;
     const int i_tok = valid ? R / G : 0;
     const int g = valid ? R - i_tok * G : 0;
-    const int vis = valid ? C + i_tok + 1 : 0;              // keys this row sees
+    // keys this row sees; rows past the sequence are computed like the piece's last row and
+    // dropped (with 0 here they would take the masking path on every tile and slow their group)
+    const int vis = valid ? C + i_tok + 1 : kv_cap;
     const size_t row_off = ((size_t)(tok0 + i_tok) * p.Hq + (size_t)it.kvh * G + g) * D;
     if (dual || st == 0) {
       // ---- Q row -> shared memory (swizzled), zero for rows past the sequence
@@ -624,6 +627,61 @@ __global__ void __launch_bounds__(128) prefill_merge_kernel(const Params p) {
 }
 
 // ------------------------------------------------------------------ host side
+namespace {
+// Relative cost of a CTA in tenths of a microsecond, as measured on B200: a 128-key tile
+// with two query tiles is bound by the softmax / tensor pipeline, with one by its K/V
+// bytes; every CTA pays for its set-up, query load, pipeline fill and epilogue; a split
+// adds the partials' round trip and the merge launch.
+constexpr long long COST_TILE_DUAL = 21, COST_TILE_SINGLE = 15, COST_CTA = 100, COST_PARTIAL = 8, COST_MERGE = 80;
+
+int sm_count() {
+  static int cached = 0;
+  if (cached > 0) return cached;
+  int dev = 0, n = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess ||
+      cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || n <= 0) {
+    cudaGetLastError();                                      // no device here: plan for a B200
+    return 148;
+  }
+  return cached = n;
+}
+
+// Finish time of the launch if the K/V range of every sequence is cut into chunks of
+// `chunk_tiles` tiles: the hardware hands CTAs, longest first, to whichever SM is free.
+long long estimate_makespan(const efim_cache_desc* c, const efim_batch_desc* b, long long chunk_tiles, int n_sm) {
+  const int G = c->num_q_heads / c->num_kv_heads;
+  std::vector<long long> cost;
+  bool split = false;
+  for (int s = 0; s < b->batch; ++s) {
+    const long long N = b->h_new_len[s], C = b->h_cached_len[s];
+    if (N <= 0) continue;
+    const long long rows = N * G;
+    const long long kt_max = (C + N + BN - 1) / BN;
+    long long S = std::max<long long>(1, std::min<long long>(16, (kt_max + chunk_tiles - 1) / chunk_tiles));
+    const long long ct = (kt_max + S - 1) / S;
+    S = (kt_max + ct - 1) / ct;
+    split |= S > 1;
+    for (long long row0 = 0; row0 < rows; row0 += NQ * BM) {
+      const long long rows_here = std::min<long long>(rows - row0, NQ * BM);
+      const long long kt = (C + (row0 + rows_here - 1) / G + 1 + BN - 1) / BN;
+      const long long tc = rows_here > BM ? COST_TILE_DUAL : COST_TILE_SINGLE;
+      for (long long tb = 0; tb < kt; tb += ct)
+        cost.insert(cost.end(), (size_t)c->num_kv_heads,
+                    COST_CTA + std::min(ct, kt - tb) * tc + (S > 1 ? COST_PARTIAL : 0));
+    }
+  }
+  std::sort(cost.begin(), cost.end(), std::greater<long long>());
+  std::vector<long long> sm((size_t)n_sm, 0);                // min-heap of SM finish times
+  auto later = std::greater<long long>();
+  for (long long x : cost) {
+    std::pop_heap(sm.begin(), sm.end(), later);
+    sm.back() += x;
+    std::push_heap(sm.begin(), sm.end(), later);
+  }
+  return *std::max_element(sm.begin(), sm.end()) + (split ? COST_MERGE : 0);
+}
+}  // namespace
+
 Plan make_plan(const efim_cache_desc* c, const efim_batch_desc* b, WorkItem* items, int32_t* split_tokens) {
   const int G = c->num_q_heads / c->num_kv_heads;
   const int Hkv = c->num_kv_heads;
@@ -640,11 +698,19 @@ Plan make_plan(const efim_cache_desc* c, const efim_batch_desc* b, WorkItem* ite
       tiles_total += kt * Hkv;
     }
   }
-  // Few long items cannot fill 148 SMs: cut the KV range of a sequence into chunks so
-  // that there are about two CTAs per SM, each at least 4 KV tiles long.
-  const long long want_ctas = 148 * 2;
+  // Few long items cannot fill the SMs, or leave a ragged last wave: try cutting the K/V
+  // range of every sequence into chunks that give about 1, 2, 3 or 4 CTAs per SM (each at
+  // least 4 tiles long) and keep the cut, or none, with the earliest estimated finish.
+  const int n_sm = sm_count();
   long long chunk_tiles = 1LL << 40;
-  if (n_unsplit < want_ctas && tiles_total > 0) chunk_tiles = std::max<long long>(4, (tiles_total + want_ctas - 1) / want_ctas);
+  if (n_unsplit < 4LL * n_sm && tiles_total > 0) {
+    long long best = estimate_makespan(c, b, chunk_tiles, n_sm);
+    for (int k = 1; k <= 4; ++k) {
+      const long long ct = std::max<long long>(4, (tiles_total + (long long)n_sm * k - 1) / ((long long)n_sm * k));
+      const long long t = estimate_makespan(c, b, ct, n_sm);
+      if (t < best) { best = t; chunk_tiles = ct; }
+    }
+  }
   Plan pl{};
   int s_max = 1;
   long long n_items = 0;

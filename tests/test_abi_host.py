@@ -103,15 +103,19 @@ def _batch_desc(cached, new, max_pages):
 
 def test_prefill_planner_splits_few_long_items_and_not_many_short_ones():
     """Host planning of efim_append_prefill_attn, seen through its two queries: few long
-    work items get their key range split (partials + a merge launch), many items do not."""
+    work items get their key range split (partials + a merge launch) when that is estimated to
+    finish sooner; a nearly full wave and many items do not."""
     lib = efim.load_library()
     cache = _cache_desc(Hq=32, Hkv=8)
-    # cfg4a-like: 8 sequences x 8 kv heads x 2 row tiles = 128 items of 65 key tiles -> split
-    few = _batch_desc([8192] * 8, [128] * 8, 600)
+    # 2 sequences x 8 kv heads x 2 row tiles = 32 items of 65 key tiles cannot fill 148 SMs -> split
+    few = _batch_desc([8192] * 2, [128] * 2, 600)
     assert lib.efim_prefill_launch_count(ctypes.byref(cache), ctypes.byref(few)) == 2
     ws_few = lib.efim_prefill_workspace_bytes(ctypes.byref(cache), ctypes.byref(few))
-    rows = 8 * 128 * 32
+    rows = 2 * 128 * 32
     assert ws_few > rows * 128 * 4 * 2            # room for at least two fp32 partials per (token, head)
+    # cfg4a-like: 128 such items nearly fill one wave; cutting them would only add a ragged wave and a merge
+    wave = _batch_desc([8192] * 8, [128] * 8, 600)
+    assert lib.efim_prefill_launch_count(ctypes.byref(cache), ctypes.byref(wave)) == 1
     # cfg4b-like: 3200 items -> one launch, workspace is just the work list
     many = _batch_desc([5120] * 8, [3200] * 8, 600)
     assert lib.efim_prefill_launch_count(ctypes.byref(cache), ctypes.byref(many)) == 1
