@@ -189,6 +189,65 @@ efim_status efim_decode_attn_static(const efim_cache_desc* cache, int32_t batch,
                                     const void* d_q, void* d_out, float* d_lse, float sm_scale,
                                     int32_t* d_status, void* stream);
 
+/* ------------------------------------------------------------------------------------
+ * Host-side front end (no GPU work): what turns a stream of infilling requests into the
+ * (cached_len, new_len, block table) triples the three calls above consume.
+ *
+ * 1. Prompt transformation, Sec. 3.1 (Fig. 7, steps 1-5).  A per-user session keeps the
+ *    prefix and suffix as they were laid out in the user's last prompt.  For a request
+ *    (user, prefix, suffix), all token ids:
+ *      - no session (step 2):                    `<P>prefix<S>suffix<M>`, session created
+ *      - prefix = session prefix + inc, inc not empty (step 4):
+ *                                                `<P>session prefix<S>suffix<M>inc`  (EFIM, Sec. 1)
+ *        the session keeps its prefix (so the next turn's prompt again starts with the same
+ *        tokens) and takes the request's suffix
+ *      - prefix unchanged (step 5, or a repeat): `<P>prefix<S>suffix<M>`, session takes the suffix
+ *      - prefix edited or shortened:             `<P>prefix<S>suffix<M>`, session replaced
+ *    `rebase_inc_tokens` > 0 bounds inc: a longer increment is folded back into the prefix
+ *    with one PSM prompt (the paper states no bound; 0 = never).
+ * 2. Cross-request KV reuse as Sec. 1 states it: the KV of a prompt can be reused for the
+ *    tokens whose whole token prefix equals an earlier sequence's.  Reuse is per page:
+ *    admit() pins the longest run of cached full pages at the start of the prompt (leaving at
+ *    least one token to compute) and takes pages for the rest plus `reserve_tokens` of decode
+ *    room - the lowest-numbered free page first, else the least recently used unpinned cached
+ *    page (among equals the deepest one); finish() registers the full pages of the finished
+ *    sequence, frees duplicates, the partial last page and unused room.
+ * All pointers are HOST pointers; a front end is not thread safe; nothing here touches CUDA.
+ */
+typedef struct efim_frontend efim_frontend;
+
+/* values of *format */
+#define EFIM_FMT_PSM_NEW     0
+#define EFIM_FMT_EFIM        1
+#define EFIM_FMT_PSM_SUFFIX  2
+#define EFIM_FMT_PSM_SAME    3
+#define EFIM_FMT_PSM_RESET   4
+#define EFIM_FMT_PSM_REBASE  5
+
+/* NULL if num_pages <= 0 or page_size <= 0. */
+efim_frontend* efim_frontend_create(int32_t tok_p, int32_t tok_s, int32_t tok_m, int32_t rebase_inc_tokens,
+                                    int32_t num_pages, int32_t page_size);
+void efim_frontend_destroy(efim_frontend* fe);
+
+/* Builds the prompt for one request.  Needs capacity >= prefix_len + suffix_len + 3, else
+ * EFIM_ERR_OUT_OF_RANGE (and the session is left as it was). */
+efim_status efim_frontend_transform(efim_frontend* fe, int64_t user, const int32_t* h_prefix, int32_t prefix_len,
+                                    const int32_t* h_suffix, int32_t suffix_len, int32_t* h_prompt,
+                                    int32_t capacity, int32_t* prompt_len, int32_t* format, int32_t* inc_len);
+
+/* Admits a prompt: *cached_len tokens are already in the pages named by the first entries of
+ * h_block_table_row, *num_pages_out entries are written in all (ceil((prompt_len + reserve_tokens)
+ * / page_size)); the rest of the row is set to -1.  EFIM_ERR_OUT_OF_RANGE if the row is too
+ * short, EFIM_ERR_WORKSPACE if the pool has no page left to take (nothing is pinned then). */
+efim_status efim_frontend_admit(efim_frontend* fe, const int32_t* h_prompt, int32_t prompt_len,
+                                int32_t reserve_tokens, int32_t* h_block_table_row, int32_t max_pages_per_seq,
+                                int32_t* cached_len, int32_t* num_pages_out, int64_t* handle);
+/* The request is over; h_tokens[0..total_len) is the sequence whose KV its pages now hold
+ * (the prompt followed by what was generated).  EFIM_ERR_INVALID_ARG for an unknown handle. */
+efim_status efim_frontend_finish(efim_frontend* fe, int64_t handle, const int32_t* h_tokens, int32_t total_len);
+/* h_out[0..4) = prompt tokens admitted, of which found cached, pages evicted, pages free now. */
+void efim_frontend_stats(const efim_frontend* fe, int64_t* h_out);
+
 #ifdef __cplusplus
 }
 #endif

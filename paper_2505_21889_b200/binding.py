@@ -38,7 +38,9 @@ EXPORTS = ("efim_last_cuda_error", "efim_strerror", "efim_version", "efim_rope_t
            "efim_prefill_workspace_bytes", "efim_append_prefill_attn",
            "efim_decode_workspace_bytes", "efim_decode_attn",
            "efim_decode_static_scratch_bytes", "efim_decode_attn_static",
-           "efim_prefill_launch_count", "efim_decode_launch_count")
+           "efim_prefill_launch_count", "efim_decode_launch_count",
+           "efim_frontend_create", "efim_frontend_destroy", "efim_frontend_transform", "efim_frontend_admit",
+           "efim_frontend_finish", "efim_frontend_stats")
 
 
 def library_path() -> str:
@@ -84,6 +86,20 @@ def load_library():
     lib.efim_decode_attn_static.restype = ctypes.c_int
     lib.efim_decode_attn_static.argtypes = [POINTER(_CacheDesc), c_int32, c_void_p, c_int32, c_void_p, c_int32,
                                             c_void_p, c_void_p, c_void_p, c_float, c_void_p, c_void_p]
+    lib.efim_frontend_create.restype = c_void_p
+    lib.efim_frontend_create.argtypes = [c_int32, c_int32, c_int32, c_int32, c_int32, c_int32]
+    lib.efim_frontend_destroy.restype = None
+    lib.efim_frontend_destroy.argtypes = [c_void_p]
+    lib.efim_frontend_transform.restype = ctypes.c_int
+    lib.efim_frontend_transform.argtypes = [c_void_p, ctypes.c_int64, c_void_p, c_int32, c_void_p, c_int32, c_void_p,
+                                            c_int32, c_void_p, c_void_p, c_void_p]
+    lib.efim_frontend_admit.restype = ctypes.c_int
+    lib.efim_frontend_admit.argtypes = [c_void_p, c_void_p, c_int32, c_int32, c_void_p, c_int32, c_void_p, c_void_p,
+                                        c_void_p]
+    lib.efim_frontend_finish.restype = ctypes.c_int
+    lib.efim_frontend_finish.argtypes = [c_void_p, ctypes.c_int64, c_void_p, c_int32]
+    lib.efim_frontend_stats.restype = None
+    lib.efim_frontend_stats.argtypes = [c_void_p, c_void_p]
     _LIB = lib
     return lib
 
@@ -233,3 +249,60 @@ def efim_prefill_launch_count(cache: Cache, batch: Batch) -> int:
 
 def efim_decode_launch_count(cache: Cache, batch: int, max_ctx_len: int) -> int:
     return int(load_library().efim_decode_launch_count(ctypes.byref(cache.desc), batch, max_ctx_len))
+
+
+class Frontend:
+    """The host-side front end of include/efim.h (prompt transformation of Sec. 3.1 and
+    page-granular cross-request KV reuse); every method is one C call on numpy arrays."""
+
+    def __init__(self, tok_p, tok_s, tok_m, num_pages, page_size=16, rebase_inc_tokens=0):
+        self._lib = load_library()
+        self._fe = self._lib.efim_frontend_create(tok_p, tok_s, tok_m, rebase_inc_tokens, num_pages, page_size)
+        if not self._fe:
+            raise EfimError(1, "efim_frontend_create")
+        self.page_size = page_size
+
+    def close(self):
+        if self._fe:
+            self._lib.efim_frontend_destroy(self._fe)
+            self._fe = None
+
+    def __del__(self):
+        self.close()
+
+    def transform(self, user, prefix, suffix):
+        """-> (prompt int32 array, format, inc_len)."""
+        prefix = np.ascontiguousarray(prefix, np.int32)
+        suffix = np.ascontiguousarray(suffix, np.int32)
+        out = np.empty(len(prefix) + len(suffix) + 3, np.int32)
+        n, fmt, inc = c_int32(), c_int32(), c_int32()
+        st = self._lib.efim_frontend_transform(self._fe, int(user), prefix.ctypes.data, len(prefix),
+                                               suffix.ctypes.data, len(suffix), out.ctypes.data, len(out),
+                                               ctypes.addressof(n), ctypes.addressof(fmt), ctypes.addressof(inc))
+        if st != 0:
+            raise EfimError(st, "efim_frontend_transform")
+        return out[:n.value], fmt.value, inc.value
+
+    def admit(self, prompt, reserve_tokens, block_table_row):
+        """Fills `block_table_row` (int32 numpy row) -> (handle, cached_len, pages used)."""
+        prompt = np.ascontiguousarray(prompt, np.int32)
+        assert block_table_row.dtype == np.int32 and block_table_row.flags.c_contiguous
+        cached, npages, handle = c_int32(), c_int32(), ctypes.c_int64()
+        st = self._lib.efim_frontend_admit(self._fe, prompt.ctypes.data, len(prompt), int(reserve_tokens),
+                                           block_table_row.ctypes.data, len(block_table_row),
+                                           ctypes.addressof(cached), ctypes.addressof(npages),
+                                           ctypes.addressof(handle))
+        if st != 0:
+            raise EfimError(st, "efim_frontend_admit")
+        return handle.value, cached.value, npages.value
+
+    def finish(self, handle, tokens):
+        tokens = np.ascontiguousarray(tokens, np.int32)
+        st = self._lib.efim_frontend_finish(self._fe, int(handle), tokens.ctypes.data, len(tokens))
+        if st != 0:
+            raise EfimError(st, "efim_frontend_finish")
+
+    def stats(self):
+        out = np.zeros(4, np.int64)
+        self._lib.efim_frontend_stats(self._fe, out.ctypes.data)
+        return dict(prompt_tokens=int(out[0]), hit_tokens=int(out[1]), evictions=int(out[2]), free_pages=int(out[3]))
