@@ -14,3 +14,4 @@ __all__ = [
     "f32_to_bf16_bits", "bf16_bits_to_f32", "pool_bits_np", "pool_fill_torch",
     "Workload", "make_workload", "WORKLOAD_NAMES",
 ]
+from .sessions import token_tables, infill_sessions, TOK_P, TOK_S, TOK_M  # noqa: F401,E402
