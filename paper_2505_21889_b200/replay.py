@@ -58,17 +58,25 @@ def _timed(fn):
     return e0, e1
 
 
-def run_scheme(scheme, sessions, layer, pool_pages, max_pages_per_seq, observe=None, batch_size=None):
+def run_scheme(scheme, sessions, layer, pool_pages, max_pages_per_seq, observe=None, batch_size=None, graph=False,
+               shuffle_seed=None):
     """Replays all rounds under one scheme; in every round the users are served in batches of
     `batch_size` (default: all at once).  `observe(round, users, prompts, cached, bt, out,
-    dec_out)` is called after every batch (for tests).  Returns totals."""
+    dec_out)` is called after every batch (for tests).  With `graph` the decode steps of a
+    batch (two or three small launches per token) are captured into one CUDA graph and
+    replayed, which takes the host's launch pace out of the decode time.  `shuffle_seed` serves
+    the users of a round in a seeded random order instead of 0, 1, 2, ... (closed-loop clients
+    do not come back in lockstep; a fixed cyclic order is the worst case for LRU).  Returns totals."""
     assert scheme in SCHEMES
     n_users, rounds = len(sessions), len(sessions[0])
     batch_size = batch_size or n_users
     fe = efim.Frontend(TOK_P, TOK_S, TOK_M, pool_pages)
     events, totals = [], dict(prompt_tokens=0, computed_tokens=0, hit_tokens=0, evictions=0, decode_tokens=0)
+    order_rng = np.random.default_rng([shuffle_seed, 41]) if shuffle_seed is not None else None
+    orders = [order_rng.permutation(n_users).tolist() if order_rng is not None else list(range(n_users))
+              for _ in range(rounds)]
     for r, first in ((r, f) for r in range(rounds) for f in range(0, n_users, batch_size)):
-        group = list(range(first, min(n_users, first + batch_size)))
+        group = orders[r][first:first + batch_size]
         users = len(group)
         if scheme == "none":                     # nothing survives from round to round
             totals["evictions"] += fe.stats()["evictions"]
@@ -105,17 +113,28 @@ def run_scheme(scheme, sessions, layer, pool_pages, max_pages_per_seq, observe=N
         max_ctx = int(plen.max()) + steps
         dws = torch.empty(max(efim.efim_decode_workspace_bytes(layer.cache, users, max_ctx), 256), dtype=torch.uint8,
                           device=layer.device)
-        dec_out = None
-        for s in range(steps):
-            dq, dk, dv = layer.qkv([sessions[g][r]["gen"][s] for g in group])
-            sb = efim.Batch(ctx, one, d_bt, layer.device)
-            ctx = ctx + 1
-            d_ctx = torch.from_numpy(ctx).to(layer.device)
-            dec_out = torch.empty_like(dq)
-            events.append(("decode",) + _timed(lambda: (
-                efim.efim_kv_append(layer.cache, sb, layer.rope, dq, dk, dv, layer.status),
-                efim.efim_decode_attn(layer.cache, users, d_ctx, max_ctx, d_bt, dq, dec_out, None, 0.0, dws,
-                                      layer.status))))
+        # per-step inputs are laid out up front so that the loop below only enqueues kernels
+        gen_ids = np.array([[sessions[g][r]["gen"][s] for g in group] for s in range(steps)]).reshape(-1)
+        dq_all, dk_all, dv_all = (x.view(steps, users, *x.shape[1:]) for x in layer.qkv(gen_ids))
+        dec_all = torch.empty_like(dq_all)
+        step_batches = [efim.Batch(ctx + s, one, d_bt, layer.device) for s in range(steps)]
+        d_ctx_all = torch.from_numpy(np.stack([ctx + s + 1 for s in range(steps)])).to(layer.device)
+
+        def decode_loop():
+            for s in range(steps):
+                efim.efim_kv_append(layer.cache, step_batches[s], layer.rope, dq_all[s], dk_all[s], dv_all[s],
+                                    layer.status)
+                efim.efim_decode_attn(layer.cache, users, d_ctx_all[s], max_ctx, d_bt, dq_all[s], dec_all[s], None,
+                                      0.0, dws, layer.status)
+        if graph and steps > 0:
+            g = torch.cuda.CUDAGraph()
+            torch.cuda.synchronize()
+            with torch.cuda.graph(g):
+                decode_loop()
+            events.append(("decode",) + _timed(g.replay))
+        else:
+            events.append(("decode",) + _timed(decode_loop))
+        dec_out = dec_all[steps - 1] if steps > 0 else None
         torch.cuda.synchronize()
         if observe is not None:
             observe(r, group, prompts, cached.copy(), bt.copy(), out, dec_out)
@@ -145,6 +164,8 @@ def main():
     ap.add_argument("--batch-size", type=int, default=16, help="users served together (the rest wait their turn)")
     ap.add_argument("--heads", type=int, nargs=2, default=(32, 8), metavar=("HQ", "HKV"))
     ap.add_argument("--seed", type=int, default=0)
+    ap.add_argument("--in-order", action="store_true", help="serve users 0, 1, 2, ... in every round (default: seeded random order)")
+    ap.add_argument("--graph", action="store_true", help="replay each batch's decode steps as one CUDA graph")
     ap.add_argument("--schemes", nargs="+", default=list(SCHEMES), choices=SCHEMES)
     a = ap.parse_args()
     vocab = 4096
@@ -155,9 +176,10 @@ def main():
     layer = Layer(a.seed, vocab, a.heads[0], a.heads[1], 128, a.pool_pages, longest + 1)
     base = None
     for scheme in a.schemes:
-        run_scheme(scheme, [u[:1] for u in sessions], layer, a.pool_pages, max_pages)        # warm-up
-        t = run_scheme(scheme, sessions, layer, a.pool_pages, max_pages, batch_size=a.batch_size)
-        t.update(scheme=scheme, users=a.users, rounds=a.rounds, pool_pages=a.pool_pages, batch_size=a.batch_size,
+        run_scheme(scheme, [u[:1] for u in sessions], layer, a.pool_pages, max_pages, batch_size=a.batch_size)   # warm-up
+        t = run_scheme(scheme, sessions, layer, a.pool_pages, max_pages, batch_size=a.batch_size, graph=a.graph,
+                       shuffle_seed=None if a.in_order else a.seed)
+        t.update(scheme=scheme, users=a.users, rounds=a.rounds, pool_pages=a.pool_pages, batch_size=a.batch_size, graph=a.graph,
                  avg_input_tokens=t["prompt_tokens"] / (a.users * a.rounds), layer_ms=t["prefill_ms"] + t["decode_ms"])
         if scheme == "none":
             base = t["layer_ms"]

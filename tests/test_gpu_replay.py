@@ -34,8 +34,8 @@ def _full_recompute(layer_bits, prompt, gen):
     return o, od
 
 
-@pytest.mark.parametrize("scheme", ["efim", "fim"])
-def test_replay_with_reuse_equals_full_recompute(scheme):
+@pytest.mark.parametrize("scheme,graph", [("efim", False), ("fim", False), ("efim", True)])
+def test_replay_with_reuse_equals_full_recompute(scheme, graph):
     import tests.gpu_harness as H
     from paper_2505_21889_b200 import replay
     sessions = infill_sessions(5, users=3, rounds=3, vocab=VOCAB, prefix0=(60, 140), suffix0=(30, 80),
@@ -59,7 +59,7 @@ def test_replay_with_reuse_equals_full_recompute(scheme):
                 assert cached[u] >= (len(t0["prefix"]) + len(t0["suffix"]) + 3) // 16 * 16
         seen.append(cached.copy())
 
-    totals = replay.run_scheme(scheme, sessions, layer, 256, -(-longest // 16), observe)
+    totals = replay.run_scheme(scheme, sessions, layer, 256, -(-longest // 16), observe, graph=graph)
     assert len(seen) == 3 and (seen[0] == 0).all() and totals["evictions"] == 0
     assert totals["computed_tokens"] + totals["hit_tokens"] == totals["prompt_tokens"]
     if scheme == "fim":                         # the suffix follows the changed prefix: never reusable
