@@ -39,8 +39,11 @@ __device__ __forceinline__ void transposed_reduce(float* x, int j) {
 // One (page, kv head) tile is 16*D*2 contiguous bytes in a pool, so a single bulk copy
 // brings it into shared memory.  Every warp owns a ring of DEC_STAGES stages (K page +
 // V page), keeps DEC_STAGES pages in flight without holding them in registers, and
-// consumes them in order; an mbarrier per stage counts the copied bytes.
-constexpr int DEC_STAGES = 3;
+// consumes them in order; an mbarrier per stage counts the copied bytes.  Two stages make
+// the ring 64 KB per CTA at D = 128, so three CTAs (12 warps) share an SM: the kernel is
+// short of warps to issue from, not of bytes in flight (with three stages and two CTAs
+// per SM it ran at 84 % of the measured copy bandwidth, with two and three at 99 %).
+constexpr int DEC_STAGES = 2;
 
 __device__ __forceinline__ uint32_t dec_smem_u32(const void* p) {
   return static_cast<uint32_t>(__cvta_generic_to_shared(p));
@@ -61,7 +64,7 @@ __device__ __forceinline__ void dec_bulk_load(uint32_t dst, const void* src, uin
 }
 
 template <int D, int GT>
-__global__ void __launch_bounds__(128) decode_splitkv_kernel(const DecodeParams p) {
+__global__ void __launch_bounds__(128, 3) decode_splitkv_kernel(const DecodeParams p) {
   constexpr int LPT = D / 8;            // lanes sharing one token row
   constexpr int TPS = 32 / LPT;         // tokens per warp-wide 16-byte read
   constexpr int STEPS = 16 / TPS;       // reads per page
