@@ -51,15 +51,23 @@ __device__ __forceinline__ void rotate4_interleaved(uint4& v, const float* c, co
   }
 }
 
-// One CTA per new token.  Work units of the token:
-//   rotate-half: (head, j) with j < D/16 -> vectors j and j + D/16 of that head (q heads then k heads)
-//   interleaved: (head, j) with j < D/8
-//   v copy:      (kv head, j) with j < D/8
-template <int D>
-__global__ void __launch_bounds__(256) kv_append_kernel(const KvAppendParams p) {
+// WPT warps per new token, 256 threads per CTA.  A lane keeps one position along the head
+// dimension (vector j, and for the rotate-half pairing its partner j + D/16), so its
+// cos/sin values are loaded once, and walks the heads - q heads (rotated in place), then
+// k heads (rotated into the page slot) - two at a time so that several 16-byte loads are
+// in flight per lane; v is copied straight into the page slot.  Many tokens: one warp per
+// token keeps every SM full of independent streams.  Few tokens (a decode step): eight
+// warps per token, because then the time is one token's latency.
+constexpr int KV_APPEND_THREADS = 256;
+
+template <int D, int WPT>
+__global__ void __launch_bounds__(KV_APPEND_THREADS) kv_append_kernel(const KvAppendParams p) {
   constexpr int VEC = D / 8;            // 16-byte vectors per head row
   constexpr int HALF = VEC / 2;
-  const int t = blockIdx.x;
+  constexpr int LANES = 32 * WPT;       // lanes working on one token
+  const int lane = threadIdx.x % LANES;
+  const int t = blockIdx.x * (KV_APPEND_THREADS / LANES) + threadIdx.x / LANES;
+  if (t >= p.total_new_tokens) return;
   // sequence of this token: last s with q_indptr[s] <= t
   int lo = 0, hi = p.batch;
   while (hi - lo > 1) {
@@ -78,7 +86,7 @@ __global__ void __launch_bounds__(256) kv_append_kernel(const KvAppendParams p) 
     if (page < 0 || page >= p.num_pages) err = EFIM_DEV_BAD_PAGE;
   }
   if (err) {
-    if (threadIdx.x == 0 && p.status) atomicOr(p.status, err);
+    if (lane == 0 && p.status) atomicOr(p.status, err);
     return;
   }
   const int slot = pos & 15;
@@ -87,66 +95,74 @@ __global__ void __launch_bounds__(256) kv_append_kernel(const KvAppendParams p) 
   const uint4* vin = reinterpret_cast<const uint4*>(p.v_new + (size_t)t * p.Hkv * D);
   uint4* qio = p.q ? reinterpret_cast<uint4*>(p.q + (size_t)t * p.Hq * D) : nullptr;
   const int nq = p.q ? p.Hq : 0;
-
-  // v: straight copy into the page slot
-  for (int u = threadIdx.x; u < p.Hkv * VEC; u += blockDim.x) {
-    const int h = u / VEC, j = u % VEC;
-    uint4 v = ldg_stream(vin + u);
-    *reinterpret_cast<uint4*>(p.v_pool + pool_tok + (size_t)h * 16 * D + j * 8) = v;
-  }
-  if (!p.cos_sin) {
-    for (int u = threadIdx.x; u < p.Hkv * VEC; u += blockDim.x) {
-      const int h = u / VEC, j = u % VEC;
-      uint4 v = ldg_stream(kin + u);
-      *reinterpret_cast<uint4*>(p.k_pool + pool_tok + (size_t)h * 16 * D + j * 8) = v;
+  // straight copy of a [Hkv][D] row into the page slot, four vectors in flight per lane
+  auto copy_row = [&](const uint4* src, uint16_t* pool) {
+    const int n = p.Hkv * VEC;
+    for (int u0 = lane; u0 < n; u0 += 4 * LANES) {
+      uint4 v[4];
+#pragma unroll
+      for (int i = 0; i < 4; ++i)
+        if (u0 + LANES * i < n) v[i] = ldg_stream(src + u0 + LANES * i);
+#pragma unroll
+      for (int i = 0; i < 4; ++i) {
+        const int u = u0 + LANES * i;
+        if (u < n) *reinterpret_cast<uint4*>(pool + pool_tok + (size_t)(u / VEC) * 16 * D + (u % VEC) * 8) = v[i];
+      }
     }
+  };
+  copy_row(vin, p.v_pool);
+  if (!p.cos_sin) {
+    copy_row(kin, p.k_pool);
     return;
   }
   const float* cs = p.cos_sin + (size_t)pos * D;     // cos[0..D/2) then sin[0..D/2)
+  const int nh = nq + p.Hkv;
+  // where vector `vec` of head h is read from / written to
+  auto src_of = [&](int h, int vec) { return h < nq ? qio + h * VEC + vec : kin + (h - nq) * VEC + vec; };
+  auto dst_of = [&](int h, int vec) {
+    return h < nq ? qio + h * VEC + vec
+                  : reinterpret_cast<uint4*>(p.k_pool + pool_tok + (size_t)(h - nq) * 16 * D + vec * 8);
+  };
   if (!p.interleaved) {
-    const int units = (nq + p.Hkv) * HALF;
-    for (int u = threadIdx.x; u < units; u += blockDim.x) {
-      const int h = u / HALF, j = u % HALF;
-      float c[8], sn[8];
-      *reinterpret_cast<float4*>(c) = __ldg(reinterpret_cast<const float4*>(cs + j * 8));
-      *reinterpret_cast<float4*>(c + 4) = __ldg(reinterpret_cast<const float4*>(cs + j * 8 + 4));
-      *reinterpret_cast<float4*>(sn) = __ldg(reinterpret_cast<const float4*>(cs + D / 2 + j * 8));
-      *reinterpret_cast<float4*>(sn + 4) = __ldg(reinterpret_cast<const float4*>(cs + D / 2 + j * 8 + 4));
-      if (h < nq) {
-        uint4 a = qio[h * VEC + j], b = qio[h * VEC + j + HALF];
-        rotate8(a, b, c, sn);
-        qio[h * VEC + j] = a;
-        qio[h * VEC + j + HALF] = b;
-      } else {
-        const int hk = h - nq;
-        uint4 a = ldg_stream(kin + hk * VEC + j), b = ldg_stream(kin + hk * VEC + j + HALF);
-        rotate8(a, b, c, sn);
-        uint16_t* dst = p.k_pool + pool_tok + (size_t)hk * 16 * D;
-        *reinterpret_cast<uint4*>(dst + j * 8) = a;
-        *reinterpret_cast<uint4*>(dst + (j + HALF) * 8) = b;
+    constexpr int HP = LANES / HALF;                 // heads the token's lanes cover at once
+    const int j = lane % HALF, h0 = lane / HALF;
+    float c[8], sn[8];
+    *reinterpret_cast<float4*>(c) = __ldg(reinterpret_cast<const float4*>(cs + j * 8));
+    *reinterpret_cast<float4*>(c + 4) = __ldg(reinterpret_cast<const float4*>(cs + j * 8 + 4));
+    *reinterpret_cast<float4*>(sn) = __ldg(reinterpret_cast<const float4*>(cs + D / 2 + j * 8));
+    *reinterpret_cast<float4*>(sn + 4) = __ldg(reinterpret_cast<const float4*>(cs + D / 2 + j * 8 + 4));
+    for (int h = h0; h < nh; h += 2 * HP) {
+      const int h2 = h + HP;
+      uint4 a = *src_of(h, j), b = *src_of(h, j + HALF), a2, b2;
+      if (h2 < nh) { a2 = *src_of(h2, j); b2 = *src_of(h2, j + HALF); }
+      rotate8(a, b, c, sn);
+      *dst_of(h, j) = a;
+      *dst_of(h, j + HALF) = b;
+      if (h2 < nh) {
+        rotate8(a2, b2, c, sn);
+        *dst_of(h2, j) = a2;
+        *dst_of(h2, j + HALF) = b2;
       }
     }
   } else {
-    const int units = (nq + p.Hkv) * VEC;
-    for (int u = threadIdx.x; u < units; u += blockDim.x) {
-      const int h = u / VEC, j = u % VEC;
-      float c[4], sn[4];
-      *reinterpret_cast<float4*>(c) = __ldg(reinterpret_cast<const float4*>(cs + j * 4));
-      *reinterpret_cast<float4*>(sn) = __ldg(reinterpret_cast<const float4*>(cs + D / 2 + j * 4));
-      if (h < nq) {
-        uint4 a = qio[h * VEC + j];
-        rotate4_interleaved(a, c, sn);
-        qio[h * VEC + j] = a;
-      } else {
-        const int hk = h - nq;
-        uint4 a = ldg_stream(kin + hk * VEC + j);
-        rotate4_interleaved(a, c, sn);
-        *reinterpret_cast<uint4*>(p.k_pool + pool_tok + (size_t)hk * 16 * D + j * 8) = a;
+    constexpr int HP = LANES / VEC;
+    const int j = lane % VEC, h0 = lane / VEC;
+    float c[4], sn[4];
+    *reinterpret_cast<float4*>(c) = __ldg(reinterpret_cast<const float4*>(cs + j * 4));
+    *reinterpret_cast<float4*>(sn) = __ldg(reinterpret_cast<const float4*>(cs + D / 2 + j * 4));
+    for (int h = h0; h < nh; h += 2 * HP) {
+      const int h2 = h + HP;
+      uint4 a = *src_of(h, j), a2;
+      if (h2 < nh) a2 = *src_of(h2, j);
+      rotate4_interleaved(a, c, sn);
+      *dst_of(h, j) = a;
+      if (h2 < nh) {
+        rotate4_interleaved(a2, c, sn);
+        *dst_of(h2, j) = a2;
       }
     }
   }
 }
-
 }  // namespace efim
 
 extern "C" efim_status efim_rope_table_build(double base, int32_t head_dim, int32_t max_position, float* h_out) {
@@ -198,10 +214,23 @@ extern "C" efim_status efim_kv_append(const efim_cache_desc* cache, const efim_b
   p.Hq = cache->num_q_heads;
   p.Hkv = cache->num_kv_heads;
   cudaStream_t s = static_cast<cudaStream_t>(stream);
-  if (cache->head_dim == 128)
-    efim::kv_append_kernel<128><<<batch->total_new_tokens, 256, 0, s>>>(p);
-  else
-    efim::kv_append_kernel<64><<<batch->total_new_tokens, 256, 0, s>>>(p);
+  // warps per token: 1 when there are enough tokens to fill the GPU with independent warps, up to 8 for a handful
+  const int T = batch->total_new_tokens;
+  const int wpt = T >= 16384 ? 1 : T >= 4096 ? 2 : T >= 1024 ? 4 : 8;
+  const unsigned grid = (unsigned)(((long long)T * wpt * 32 + efim::KV_APPEND_THREADS - 1) / efim::KV_APPEND_THREADS);
+#define EFIM_KV_APPEND_LAUNCH(D_, W_) efim::kv_append_kernel<D_, W_><<<grid, efim::KV_APPEND_THREADS, 0, s>>>(p)
+  if (cache->head_dim == 128) {
+    if (wpt == 1) EFIM_KV_APPEND_LAUNCH(128, 1);
+    else if (wpt == 2) EFIM_KV_APPEND_LAUNCH(128, 2);
+    else if (wpt == 4) EFIM_KV_APPEND_LAUNCH(128, 4);
+    else EFIM_KV_APPEND_LAUNCH(128, 8);
+  } else {
+    if (wpt == 1) EFIM_KV_APPEND_LAUNCH(64, 1);
+    else if (wpt == 2) EFIM_KV_APPEND_LAUNCH(64, 2);
+    else if (wpt == 4) EFIM_KV_APPEND_LAUNCH(64, 4);
+    else EFIM_KV_APPEND_LAUNCH(64, 8);
+  }
+#undef EFIM_KV_APPEND_LAUNCH
   EFIM_CUDA_TRY(cudaGetLastError());
   return EFIM_OK;
 }
