@@ -6,7 +6,8 @@ One "step" = one turn of one layer over one ragged batch:
     -> efim_kv_append(1 generated token per sequence) -> efim_decode_attn
 `value` = new tokens (inc + generated) that went through the path per second, inputs
 resident in HBM; `e2e` = the same with the step's q/k/v coming from pinned host
-memory and the outputs copied back, copies inside the timed region.
+memory and the outputs copied back, copies inside the timed region (pipelined over
+three streams: the copies of neighbouring steps run beside a step's kernels).
 
     python bench.py [--gpus N] [--steps K] [--warmup W] [--workload cfg2] [--impl reference]
 
@@ -299,17 +300,20 @@ def run_native(args):
     def ev():
         return torch.cuda.Event(enable_timing=True)
 
-    def step(marks=None):
-        """The four calls of one turn on the current stream; marks = 5 events or None."""
+    def step(marks=None, io=None):
+        """The four calls of one turn on the current stream; marks = 5 events or None;
+        io = another set of input/output tensors (q, k, v, out, dq, dk, dv, dout) or None."""
+        q_, k_, v_, out_, dq_, dk_, dv_, dout_ = io if io else (
+            q, k_new, v_new, out, *((dq, dk, dv, dout) if has_decode else (None,) * 4))
         if marks: marks[0].record(stream)
-        efim.efim_kv_append(cache, batch, rope, q, k_new, v_new, status)
+        efim.efim_kv_append(cache, batch, rope, q_, k_, v_, status)
         if marks: marks[1].record(stream)
-        efim.efim_append_prefill_attn(cache, batch, q, out, None, 0.0, ws_p, status)
+        efim.efim_append_prefill_attn(cache, batch, q_, out_, None, 0.0, ws_p, status)
         if marks: marks[2].record(stream)
         if has_decode:
-            efim.efim_kv_append(cache, dec_batch, rope, dq, dk, dv, status)
+            efim.efim_kv_append(cache, dec_batch, rope, dq_, dk_, dv_, status)
             if marks: marks[3].record(stream)
-            efim.efim_decode_attn(cache, B, d_ctx, max_ctx, batch.d_block_table, dq, dout, None, 0.0, ws_d, status)
+            efim.efim_decode_attn(cache, B, d_ctx, max_ctx, batch.d_block_table, dq_, dout_, None, 0.0, ws_d, status)
         elif marks:
             marks[3].record(stream)
         if marks: marks[4].record(stream)
@@ -320,18 +324,55 @@ def run_native(args):
             dq.copy_(dq0)
         flush.fill_(1)                         # evict L2 between timed steps
 
-    def e2e_step():
-        q.copy_(h_q.view(torch.bfloat16), non_blocking=True)
-        k_new.copy_(h_k.view(torch.bfloat16), non_blocking=True)
-        v_new.copy_(h_v.view(torch.bfloat16), non_blocking=True)
-        if has_decode:
-            dq.copy_(h_dq.view(torch.bfloat16), non_blocking=True)
-            dk.copy_(h_dk.view(torch.bfloat16), non_blocking=True)
-            dv.copy_(h_dv.view(torch.bfloat16), non_blocking=True)
-        step()
-        h_out.copy_(out.view(torch.int16), non_blocking=True)
-        if has_decode:
-            h_dout.copy_(dout.view(torch.int16), non_blocking=True)
+    # End to end: every step's q/k/v come from pinned host memory and its outputs go back to
+    # pinned host memory.  The copies of step i+1 and i-1 run on their own streams beside the
+    # kernels of step i (two sets of device and host buffers), as a serving loop would do it;
+    # all of them lie inside the timed region.
+    s_in, s_out = torch.cuda.Stream(), torch.cuda.Stream()
+    io_sets, h_outs = [], []
+    for _ in range(2):
+        d = (torch.empty_like(q), torch.empty_like(k_new), torch.empty_like(v_new), torch.empty_like(out))
+        d += (torch.empty_like(dq), torch.empty_like(dk), torch.empty_like(dv), torch.empty_like(dout)) \
+            if has_decode else (None,) * 4
+        io_sets.append(d)
+        h_outs.append((torch.empty(out.shape, dtype=torch.int16).pin_memory(),
+                       torch.empty(dout.shape, dtype=torch.int16).pin_memory() if has_decode else None))
+    h_ins = (h_q, h_k, h_v) + ((h_dq, h_dk, h_dv) if has_decode else ())
+
+    def e2e_run(n):
+        """n pipelined steps; returns (start, end) events that bracket all copies and kernels."""
+        t0, t1 = ev(), ev()
+        in_done = [None, None]
+        comp_done = [None, None]
+        out_done = [None, None]
+        s_in.wait_stream(stream)
+        s_out.wait_stream(stream)
+        t0.record(stream)
+        s_in.wait_event(t0)
+        for i in range(n):
+            b = i & 1
+            io = io_sets[b]
+            with torch.cuda.stream(s_in):
+                if comp_done[b] is not None:
+                    s_in.wait_event(comp_done[b])          # the kernels of step i-2 are done with these inputs
+                for dst, src in zip((io[0], io[1], io[2], io[4], io[5], io[6]), h_ins):
+                    dst.copy_(src.view(torch.bfloat16), non_blocking=True)
+                in_done[b] = ev(); in_done[b].record(s_in)
+            stream.wait_event(in_done[b])
+            if out_done[b] is not None:
+                stream.wait_event(out_done[b])             # step i-2's outputs have left the device
+            step(io=io)
+            comp_done[b] = ev(); comp_done[b].record(stream)
+            with torch.cuda.stream(s_out):
+                s_out.wait_event(comp_done[b])
+                h_outs[b][0].copy_(io[3].view(torch.int16), non_blocking=True)
+                if has_decode:
+                    h_outs[b][1].copy_(io[7].view(torch.int16), non_blocking=True)
+                out_done[b] = ev(); out_done[b].record(s_out)
+        stream.wait_stream(s_in)
+        stream.wait_stream(s_out)
+        t1.record(stream)
+        return t0, t1
 
     # launches of our kernels per step, as the library plans them
     launches = 1 + efim.efim_prefill_launch_count(cache, batch)
@@ -359,19 +400,12 @@ def run_native(args):
     step_ms = np.array([m[0].elapsed_time(m[4]) for m in marks])
     local_ms = float(step_ms.sum())
     # ---------------- end to end (host buffers)
-    for _ in range(2):
-        flush.fill_(1)
-        e2e_step()
+    e2e_run(3)
     barrier()
-    e2e_marks = [(ev(), ev()) for _ in range(args.steps)]
-    for a, b in e2e_marks:
-        flush.fill_(1)
-        a.record(stream)
-        e2e_step()
-        b.record(stream)
+    e2e_t0, e2e_t1 = e2e_run(args.steps)
     barrier()
     clocks = sampler.stop()
-    e2e_ms = float(sum(a.elapsed_time(b) for a, b in e2e_marks))
+    e2e_ms = float(e2e_t0.elapsed_time(e2e_t1))
     if int(status.item()) != 0:
         raise RuntimeError(f"device status word {int(status.item()):#x} after the run")
 
@@ -440,7 +474,8 @@ def run_native(args):
                    "parallelism": f"replicas x{world}"},
         "clocks": clocks,
         "e2e": {"value": job_tokens / (job_e2e_ms / 1e3), "unit": UNIT,
-                "h2d_bytes_per_step": int(h2d), "d2h_bytes_per_step": int(d2h)},
+                "h2d_bytes_per_step": int(h2d), "d2h_bytes_per_step": int(d2h),
+                "overlap": "copies of steps i+1 and i-1 on their own streams beside the kernels of step i"},
         "gpu_launches": launches * args.steps,
         "breakdown": breakdown,
         "roofline": roof,
