@@ -216,3 +216,32 @@ def test_run_to_run_bit_reproducible():
         torch.cuda.synchronize()
         outs.append((H.torch_to_bits(dw.out), dw.lse.cpu().numpy()))
     assert np.array_equal(outs[0][0], outs[1][0]) and np.array_equal(outs[0][1], outs[1][1])
+
+
+@pytest.mark.parametrize("T,Hq,Hkv,D,interleaved", [
+    (1024, 4, 2, 128, False),     # four warps per token
+    (1023, 6, 2, 64, True),       # eight warps per token, odd token count
+    (4096, 4, 4, 64, False),      # two warps per token
+    (5000, 3, 1, 128, True),      # two warps per token, heads not a multiple of the lanes' head stride
+    (16384, 2, 1, 64, False),     # one warp per token
+    (16391, 2, 2, 128, False),    # one warp per token, ragged last CTA
+])
+def test_kv_append_token_count_regimes(T, Hq, Hkv, D, interleaved):
+    """efim_kv_append picks the number of warps per token from the token count; every
+    variant must place and rotate exactly like the oracle (rows of three sequences,
+    unaligned starts)."""
+    H = _harness()
+    import paper_2505_21889_b200 as efim
+    new = [T // 3, T // 5, T - T // 3 - T // 5]
+    w = _custom(Hq, Hkv, D, [13, 0, 255], new, seed=T, extra=0)
+    dw = H.DeviceWorkload(w, interleaved=interleaved)
+    dw.gpu_kv_append()
+    torch.cuda.synchronize()
+    assert int(dw.status.item()) == 0
+    kp, vp, bt, seqs = w.compact_host_pool()
+    q_rot = orc.kv_append(kp, vp, bt, w.cached_len, w.new_len, dw.q_bits, dw.k_bits, dw.v_bits, w.rope_base,
+                          interleaved)
+    used = np.array(sorted(set(w.block_table[w.block_table >= 0].tolist())), np.int64)
+    assert np.array_equal(dw.pages_from_device("v", used), vp)            # placement and copy: bit-exact
+    H.assert_rope_close(dw.pages_from_device("k", used), kp, "k pages")
+    H.assert_rope_close(H.torch_to_bits(dw.q), q_rot, "q")
