@@ -280,6 +280,16 @@ def run_native(args):
     out = torch.empty_like(q)
     h_out = torch.empty(out.shape, dtype=torch.int16).pin_memory()
     ws_p = torch.empty(max(efim.efim_prefill_workspace_bytes(cache, batch), 256), dtype=torch.uint8, device=dev)
+    # The work list depends on the batch's lengths only, not on the layer: planned once per
+    # batch (as a model would, then run for every layer) and timed on its own.
+    plan = None
+    plan_ms = 0.0
+    if T > 0:
+        efim.efim_prefill_plan(cache, batch)
+        t_plan = time.perf_counter()
+        for _ in range(10):
+            plan = efim.efim_prefill_plan(cache, batch)
+        plan_ms = (time.perf_counter() - t_plan) / 10 * 1e3
     if has_decode:
         dqb, dkb, dvb = w.decode_qkv(0)
         h_dq = torch.from_numpy(dqb.view(np.int16)).pin_memory()
@@ -308,7 +318,7 @@ def run_native(args):
         if marks: marks[0].record(stream)
         efim.efim_kv_append(cache, batch, rope, q_, k_, v_, status)
         if marks: marks[1].record(stream)
-        efim.efim_append_prefill_attn(cache, batch, q_, out_, None, 0.0, ws_p, status)
+        efim.efim_append_prefill_attn(cache, batch, q_, out_, None, 0.0, ws_p, status, plan=plan)
         if marks: marks[2].record(stream)
         if has_decode:
             efim.efim_kv_append(cache, dec_batch, rope, dq_, dk_, dv_, status)
@@ -422,6 +432,7 @@ def run_native(args):
     kv_bytes = cnt["kv_append_bytes_per_token"] * cnt["new_tokens"]
     breakdown = {
         "kv_append_ms": t_app, "kv_append_gbs": kv_bytes / t_app / 1e6,
+        "prefill_plan_host_ms": plan_ms,       # once per batch, outside the step (amortised over a model's layers)
         "append_prefill_ms": t_pre, "append_prefill_tflops": cnt["prefill_flops"] / t_pre / 1e9,
         "append_prefill_kv_gbs": cnt["prefill_kv_bytes"] / t_pre / 1e6,
         "decode_kv_append_ms": t_app1, "decode_ms": t_dec,

@@ -138,6 +138,27 @@ efim_status efim_append_prefill_attn(const efim_cache_desc* cache, const efim_ba
                                      int32_t* d_status, void* stream);
 
 /*
+ * Step 2 with the planning taken out of the call.  The work list depends only on the batch's
+ * lengths and the cache shape, not on the layer: a model runs step 2 once per layer on the
+ * same batch, so it plans once and runs many times.  efim_prefill_plan() writes the plan - a
+ * relocatable blob of efim_prefill_plan_bytes() bytes - into HOST memory of the caller;
+ * efim_append_prefill_attn_planned() is efim_append_prefill_attn() with that blob in place of
+ * the planning (same results bit for bit, same workspace size).  The blob's lists are copied
+ * to the workspace on `stream` in every call: keep the blob alive and unchanged until the
+ * stream has passed the call (pinned memory makes the copy asynchronous).
+ * EFIM_ERR_INVALID_ARG if the blob was not made for this cache shape and these lengths
+ * (checked against a hash of the host mirrors), EFIM_ERR_WORKSPACE if plan_bytes is too small.
+ */
+size_t efim_prefill_plan_bytes(const efim_cache_desc* cache, const efim_batch_desc* batch);
+efim_status efim_prefill_plan(const efim_cache_desc* cache, const efim_batch_desc* batch,
+                              void* h_plan, size_t plan_bytes);
+efim_status efim_append_prefill_attn_planned(const efim_cache_desc* cache, const efim_batch_desc* batch,
+                                             const void* h_plan, size_t plan_bytes,
+                                             const void* d_q, void* d_out, float* d_lse, float sm_scale,
+                                             void* d_workspace, size_t workspace_bytes,
+                                             int32_t* d_status, void* stream);
+
+/*
  * Step 3 (decode of the generated middle, EFIM Sec. 2.2 / Fig. 4): one query
  * token per sequence over keys [0, ctx_len[s]) (ctx_len counts the token just
  * appended).  The key range is cut into fixed-length chunks; each chunk yields a

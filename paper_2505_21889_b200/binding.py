@@ -39,6 +39,7 @@ EXPORTS = ("efim_last_cuda_error", "efim_strerror", "efim_version", "efim_rope_t
            "efim_decode_workspace_bytes", "efim_decode_attn",
            "efim_decode_static_scratch_bytes", "efim_decode_attn_static",
            "efim_prefill_launch_count", "efim_decode_launch_count",
+           "efim_prefill_plan_bytes", "efim_prefill_plan", "efim_append_prefill_attn_planned",
            "efim_frontend_create", "efim_frontend_destroy", "efim_frontend_transform", "efim_frontend_admit",
            "efim_frontend_finish", "efim_frontend_stats")
 
@@ -71,6 +72,14 @@ def load_library():
     lib.efim_append_prefill_attn.restype = ctypes.c_int
     lib.efim_append_prefill_attn.argtypes = [POINTER(_CacheDesc), POINTER(_BatchDesc), c_void_p, c_void_p,
                                              c_void_p, c_float, c_void_p, c_size_t, c_void_p, c_void_p]
+    lib.efim_prefill_plan_bytes.restype = c_size_t
+    lib.efim_prefill_plan_bytes.argtypes = [POINTER(_CacheDesc), POINTER(_BatchDesc)]
+    lib.efim_prefill_plan.restype = ctypes.c_int
+    lib.efim_prefill_plan.argtypes = [POINTER(_CacheDesc), POINTER(_BatchDesc), c_void_p, c_size_t]
+    lib.efim_append_prefill_attn_planned.restype = ctypes.c_int
+    lib.efim_append_prefill_attn_planned.argtypes = [POINTER(_CacheDesc), POINTER(_BatchDesc), c_void_p, c_size_t,
+                                                     c_void_p, c_void_p, c_void_p, c_float, c_void_p, c_size_t,
+                                                     c_void_p, c_void_p]
     lib.efim_decode_workspace_bytes.restype = c_size_t
     lib.efim_decode_workspace_bytes.argtypes = [POINTER(_CacheDesc), c_int32, c_int32]
     lib.efim_decode_attn.restype = ctypes.c_int
@@ -202,12 +211,33 @@ def efim_prefill_workspace_bytes(cache: Cache, batch: Batch) -> int:
     return int(load_library().efim_prefill_workspace_bytes(ctypes.byref(cache.desc), ctypes.byref(batch.desc)))
 
 
+def efim_prefill_plan(cache: Cache, batch: Batch) -> np.ndarray:
+    """The work list of efim_append_prefill_attn for this batch as a host blob (uint8 array);
+    pass it as `plan=` to run without planning, e.g. once per layer."""
+    lib = load_library()
+    n = int(lib.efim_prefill_plan_bytes(ctypes.byref(cache.desc), ctypes.byref(batch.desc)))
+    if n == 0:
+        raise EfimError(1, "efim_prefill_plan_bytes")
+    blob = np.zeros(n, np.uint8)
+    st = lib.efim_prefill_plan(ctypes.byref(cache.desc), ctypes.byref(batch.desc), blob.ctypes.data, n)
+    if st != 0:
+        raise EfimError(st, "efim_prefill_plan")
+    return blob
+
+
 def efim_append_prefill_attn(cache: Cache, batch: Batch, q, out, lse=None, sm_scale=0.0,
-                             workspace=None, status=None, stream=None):
+                             workspace=None, status=None, stream=None, plan=None):
     nbytes = 0 if workspace is None else workspace.numel() * workspace.element_size()
-    st = load_library().efim_append_prefill_attn(ctypes.byref(cache.desc), ctypes.byref(batch.desc),
-                                                 _ptr(q), _ptr(out), _ptr(lse), float(sm_scale),
-                                                 _ptr(workspace), nbytes, _ptr(status), _stream_ptr(stream))
+    lib = load_library()
+    if plan is None:
+        st = lib.efim_append_prefill_attn(ctypes.byref(cache.desc), ctypes.byref(batch.desc),
+                                          _ptr(q), _ptr(out), _ptr(lse), float(sm_scale),
+                                          _ptr(workspace), nbytes, _ptr(status), _stream_ptr(stream))
+    else:
+        st = lib.efim_append_prefill_attn_planned(ctypes.byref(cache.desc), ctypes.byref(batch.desc),
+                                                  plan.ctypes.data, plan.nbytes, _ptr(q), _ptr(out), _ptr(lse),
+                                                  float(sm_scale), _ptr(workspace), nbytes, _ptr(status),
+                                                  _stream_ptr(stream))
     if st != 0:
         raise EfimError(st, "efim_append_prefill_attn")
 

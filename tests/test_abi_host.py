@@ -139,3 +139,23 @@ def test_decode_planner_chunks():
     # a context of one chunk needs neither workspace nor merge
     assert lib.efim_decode_launch_count(ctypes.byref(cache), 4096, 200) == 1
     assert lib.efim_decode_workspace_bytes(ctypes.byref(cache), 4096, 200) == 0
+
+
+def test_prefill_plan_blob_sizes_and_errors():
+    """efim_prefill_plan: the blob is a 256-byte head plus the work list and split sizes; a
+    buffer that is too small is refused; a batch with nothing new still gets a valid (empty) plan."""
+    lib = efim.load_library()
+    lib.efim_prefill_plan_bytes.restype = ctypes.c_size_t
+    cache = _cache_desc(Hq=32, Hkv=8)
+    many = _batch_desc([5120] * 8, [3200] * 8, 600)
+    n = lib.efim_prefill_plan_bytes(ctypes.byref(cache), ctypes.byref(many))
+    items = 8 * 8 * (3200 * 4 // 256)
+    assert 256 + items * 32 <= n < 256 + items * 32 + 1024
+    buf = np.zeros(n, np.uint8)
+    assert lib.efim_prefill_plan(ctypes.byref(cache), ctypes.byref(many), buf.ctypes.data, n) == 0
+    assert bytes(buf[:4]) == b"EFIM" and buf[256:].any()
+    assert lib.efim_prefill_plan(ctypes.byref(cache), ctypes.byref(many), buf.ctypes.data, n - 1) == 4
+    assert lib.efim_prefill_plan(ctypes.byref(cache), ctypes.byref(many), None, n) == 1
+    none = _batch_desc([100, 200], [0, 0], 32)
+    assert lib.efim_prefill_plan_bytes(ctypes.byref(cache), ctypes.byref(none)) == 256
+    assert lib.efim_prefill_plan(ctypes.byref(cache), ctypes.byref(none), buf.ctypes.data, 256) == 0

@@ -245,3 +245,31 @@ def test_kv_append_token_count_regimes(T, Hq, Hkv, D, interleaved):
     assert np.array_equal(dw.pages_from_device("v", used), vp)            # placement and copy: bit-exact
     H.assert_rope_close(dw.pages_from_device("k", used), kp, "k pages")
     H.assert_rope_close(H.torch_to_bits(dw.q), q_rot, "q")
+
+
+@pytest.mark.parametrize("name", ["cfg2", "cfg3", "cfg4a"])
+def test_planned_prefill_is_bit_identical_and_checks_its_plan(name):
+    """efim_append_prefill_attn_planned with a plan made once (as for every layer of a model)
+    gives the same bits as the call that plans inside; a plan for other lengths is refused."""
+    H = _harness()
+    import paper_2505_21889_b200 as efim
+    w = make_workload(name, small=True)
+    dw = H.DeviceWorkload(w)
+    dw.gpu_kv_append()
+    dw.gpu_prefill()
+    torch.cuda.synchronize()
+    want_out, want_lse = dw.out.clone(), dw.lse.clone()
+    plan = efim.efim_prefill_plan(dw.cache, dw.batch)
+    for _ in range(2):                                     # the same plan, run twice
+        dw.out.zero_()
+        dw.lse.zero_()
+        efim.efim_append_prefill_attn(dw.cache, dw.batch, dw.q, dw.out, dw.lse, 0.0, dw.ws, dw.status, plan=plan)
+        torch.cuda.synchronize()
+        assert int(dw.status.item()) == 0
+        assert torch.equal(dw.out.view(torch.int16), want_out.view(torch.int16)) and torch.equal(dw.lse, want_lse)
+    other = efim.Batch(w.cached_len + 1, w.new_len, dw.batch.d_block_table)
+    with pytest.raises(efim.EfimError) as e:
+        efim.efim_append_prefill_attn(dw.cache, other, dw.q, dw.out, dw.lse, 0.0, dw.ws, dw.status, plan=plan)
+    assert e.value.code == 1
+    with pytest.raises(efim.EfimError):                    # a truncated blob
+        efim.efim_append_prefill_attn(dw.cache, dw.batch, dw.q, dw.out, dw.lse, 0.0, dw.ws, dw.status, plan=plan[:64])
