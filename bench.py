@@ -283,6 +283,7 @@ def run_native(args):
     # The work list depends on the batch's lengths only, not on the layer: planned once per
     # batch (as a model would, then run for every layer) and timed on its own.
     plan = None
+    uploaded = [False]
     plan_ms = 0.0
     if T > 0:
         efim.efim_prefill_plan(cache, batch)
@@ -318,7 +319,9 @@ def run_native(args):
         if marks: marks[0].record(stream)
         efim.efim_kv_append(cache, batch, rope, q_, k_, v_, status)
         if marks: marks[1].record(stream)
-        efim.efim_append_prefill_attn(cache, batch, q_, out_, None, 0.0, ws_p, status, plan=plan)
+        efim.efim_append_prefill_attn(cache, batch, q_, out_, None, 0.0, ws_p, status, plan=plan,
+                                      lists_resident=uploaded[0])
+        uploaded[0] = True                       # the lists stay at the head of ws_p: uploaded once per batch
         if marks: marks[2].record(stream)
         if has_decode:
             efim.efim_kv_append(cache, dec_batch, rope, dq_, dk_, dv_, status)

@@ -143,9 +143,12 @@ efim_status efim_append_prefill_attn(const efim_cache_desc* cache, const efim_ba
  * same batch, so it plans once and runs many times.  efim_prefill_plan() writes the plan - a
  * relocatable blob of efim_prefill_plan_bytes() bytes - into HOST memory of the caller;
  * efim_append_prefill_attn_planned() is efim_append_prefill_attn() with that blob in place of
- * the planning (same results bit for bit, same workspace size).  The blob's lists are copied
- * to the workspace on `stream` in every call: keep the blob alive and unchanged until the
- * stream has passed the call (pinned memory makes the copy asynchronous).
+ * the planning (same results bit for bit, same workspace size).  With lists_resident = 0 the
+ * blob's lists are first copied to the head of the workspace on `stream`: keep the blob alive
+ * and unchanged until the stream has passed the call (pinned memory makes the copy
+ * asynchronous).  With lists_resident = 1 the call copies nothing and only launches: the head
+ * of this workspace must still hold the lists from an earlier call with the same plan (the
+ * kernels only read them; the partials live behind them) - upload once per batch, run per layer.
  * EFIM_ERR_INVALID_ARG if the blob was not made for this cache shape and these lengths
  * (checked against a hash of the host mirrors), EFIM_ERR_WORKSPACE if plan_bytes is too small.
  */
@@ -153,7 +156,7 @@ size_t efim_prefill_plan_bytes(const efim_cache_desc* cache, const efim_batch_de
 efim_status efim_prefill_plan(const efim_cache_desc* cache, const efim_batch_desc* batch,
                               void* h_plan, size_t plan_bytes);
 efim_status efim_append_prefill_attn_planned(const efim_cache_desc* cache, const efim_batch_desc* batch,
-                                             const void* h_plan, size_t plan_bytes,
+                                             const void* h_plan, size_t plan_bytes, int32_t lists_resident,
                                              const void* d_q, void* d_out, float* d_lse, float sm_scale,
                                              void* d_workspace, size_t workspace_bytes,
                                              int32_t* d_status, void* stream);

@@ -78,7 +78,7 @@ def load_library():
     lib.efim_prefill_plan.argtypes = [POINTER(_CacheDesc), POINTER(_BatchDesc), c_void_p, c_size_t]
     lib.efim_append_prefill_attn_planned.restype = ctypes.c_int
     lib.efim_append_prefill_attn_planned.argtypes = [POINTER(_CacheDesc), POINTER(_BatchDesc), c_void_p, c_size_t,
-                                                     c_void_p, c_void_p, c_void_p, c_float, c_void_p, c_size_t,
+                                                     c_int32, c_void_p, c_void_p, c_void_p, c_float, c_void_p, c_size_t,
                                                      c_void_p, c_void_p]
     lib.efim_decode_workspace_bytes.restype = c_size_t
     lib.efim_decode_workspace_bytes.argtypes = [POINTER(_CacheDesc), c_int32, c_int32]
@@ -226,7 +226,7 @@ def efim_prefill_plan(cache: Cache, batch: Batch) -> np.ndarray:
 
 
 def efim_append_prefill_attn(cache: Cache, batch: Batch, q, out, lse=None, sm_scale=0.0,
-                             workspace=None, status=None, stream=None, plan=None):
+                             workspace=None, status=None, stream=None, plan=None, lists_resident=False):
     nbytes = 0 if workspace is None else workspace.numel() * workspace.element_size()
     lib = load_library()
     if plan is None:
@@ -235,7 +235,8 @@ def efim_append_prefill_attn(cache: Cache, batch: Batch, q, out, lse=None, sm_sc
                                           _ptr(workspace), nbytes, _ptr(status), _stream_ptr(stream))
     else:
         st = lib.efim_append_prefill_attn_planned(ctypes.byref(cache.desc), ctypes.byref(batch.desc),
-                                                  plan.ctypes.data, plan.nbytes, _ptr(q), _ptr(out), _ptr(lse),
+                                                  plan.ctypes.data, plan.nbytes, 1 if lists_resident else 0,
+                                                  _ptr(q), _ptr(out), _ptr(lse),
                                                   float(sm_scale), _ptr(workspace), nbytes, _ptr(status),
                                                   _stream_ptr(stream))
     if st != 0:

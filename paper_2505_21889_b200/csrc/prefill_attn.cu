@@ -94,8 +94,9 @@ extern "C" efim_status efim_prefill_plan(const efim_cache_desc* cache, const efi
 }
 
 extern "C" efim_status efim_append_prefill_attn_planned(const efim_cache_desc* cache, const efim_batch_desc* batch,
-                                                        const void* h_plan, size_t plan_bytes, const void* d_q,
-                                                        void* d_out, float* d_lse, float sm_scale, void* d_workspace,
+                                                        const void* h_plan, size_t plan_bytes,
+                                                        int32_t lists_resident, const void* d_q, void* d_out,
+                                                        float* d_lse, float sm_scale, void* d_workspace,
                                                         size_t workspace_bytes, int32_t* d_status, void* stream) {
   using namespace efim;
   efim_status st = check_cache(cache);
@@ -125,8 +126,10 @@ extern "C" efim_status efim_append_prefill_attn_planned(const efim_cache_desc* c
   cudaStream_t s = static_cast<cudaStream_t>(stream);
   char* ws = static_cast<char*>(d_workspace);
   // work list + per-sequence split sizes go to the head of the workspace in one copy
-  EFIM_CUDA_TRY(cudaMemcpyAsync(ws, static_cast<const unsigned char*>(h_plan) + PLAN_HEAD_BYTES,
-                                pl.items_bytes + pl.split_bytes, cudaMemcpyHostToDevice, s));
+  // (unless an earlier call with this plan and workspace has left them there)
+  if (!lists_resident)
+    EFIM_CUDA_TRY(cudaMemcpyAsync(ws, static_cast<const unsigned char*>(h_plan) + PLAN_HEAD_BYTES,
+                                  pl.items_bytes + pl.split_bytes, cudaMemcpyHostToDevice, s));
   pf::Params p{};
   p.q = static_cast<const uint16_t*>(d_q);
   p.out = static_cast<uint16_t*>(d_out);
@@ -167,6 +170,6 @@ extern "C" efim_status efim_append_prefill_attn(const efim_cache_desc* cache, co
   const pf::Plan sized = pf::make_plan(cache, batch, nullptr, nullptr);
   std::vector<unsigned char> blob(PLAN_HEAD_BYTES + sized.items_bytes + sized.split_bytes);
   fill_plan(cache, batch, &sized, blob.data());
-  return efim_append_prefill_attn_planned(cache, batch, blob.data(), blob.size(), d_q, d_out, d_lse, sm_scale,
+  return efim_append_prefill_attn_planned(cache, batch, blob.data(), blob.size(), 0, d_q, d_out, d_lse, sm_scale,
                                           d_workspace, workspace_bytes, d_status, stream);
 }

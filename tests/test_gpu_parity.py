@@ -260,10 +260,11 @@ def test_planned_prefill_is_bit_identical_and_checks_its_plan(name):
     torch.cuda.synchronize()
     want_out, want_lse = dw.out.clone(), dw.lse.clone()
     plan = efim.efim_prefill_plan(dw.cache, dw.batch)
-    for _ in range(2):                                     # the same plan, run twice
+    for resident in (False, True, True):                   # the same plan: uploaded once, then only launched
         dw.out.zero_()
         dw.lse.zero_()
-        efim.efim_append_prefill_attn(dw.cache, dw.batch, dw.q, dw.out, dw.lse, 0.0, dw.ws, dw.status, plan=plan)
+        efim.efim_append_prefill_attn(dw.cache, dw.batch, dw.q, dw.out, dw.lse, 0.0, dw.ws, dw.status, plan=plan,
+                                      lists_resident=resident)
         torch.cuda.synchronize()
         assert int(dw.status.item()) == 0
         assert torch.equal(dw.out.view(torch.int16), want_out.view(torch.int16)) and torch.equal(dw.lse, want_lse)
