@@ -2,8 +2,8 @@
 """Benchmark of the EFIM per-turn GPU path on synthetic multi-turn infilling batches.
 
 One "step" = one turn of one layer over one ragged batch:
-    efim_kv_append(inc tokens) -> efim_append_prefill_attn
-    -> efim_kv_append(1 generated token per sequence) -> efim_decode_attn
+    efim_kv_append(inc tokens) -> efim_append_prefill_attn (planned once per batch)
+    -> efim_decode_step (kv_append of 1 generated token per sequence fused with decode attention)
 `value` = new tokens (inc + generated) that went through the path per second, inputs
 resident in HBM; `e2e` = the same with the step's q/k/v coming from pinned host
 memory and the outputs copied back, copies inside the timed region (pipelined over
@@ -323,12 +323,11 @@ def run_native(args):
                                       lists_resident=uploaded[0])
         uploaded[0] = True                       # the lists stay at the head of ws_p: uploaded once per batch
         if marks: marks[2].record(stream)
+        if marks: marks[3].record(stream)
         if has_decode:
-            efim.efim_kv_append(cache, dec_batch, rope, dq_, dk_, dv_, status)
-            if marks: marks[3].record(stream)
-            efim.efim_decode_attn(cache, B, d_ctx, max_ctx, batch.d_block_table, dq_, dout_, None, 0.0, ws_d, status)
-        elif marks:
-            marks[3].record(stream)
+            # the generated token's kv_append is fused into the decode kernel
+            efim.efim_decode_step(cache, B, d_ctx, max_ctx, batch.d_block_table, rope, dq_, dk_, dv_, dout_, None, 0.0,
+                                  ws_d, status)
         if marks: marks[4].record(stream)
 
     def reset_inputs():
@@ -390,7 +389,7 @@ def run_native(args):
     # launches of our kernels per step, as the library plans them
     launches = 1 + efim.efim_prefill_launch_count(cache, batch)
     if has_decode:
-        launches += 1 + efim.efim_decode_launch_count(cache, B, max_ctx)
+        launches += efim.efim_decode_launch_count(cache, B, max_ctx)
 
     def barrier():
         if dist is not None:
@@ -438,7 +437,7 @@ def run_native(args):
         "prefill_plan_host_ms": plan_ms,       # once per batch, outside the step (amortised over a model's layers)
         "append_prefill_ms": t_pre, "append_prefill_tflops": cnt["prefill_flops"] / t_pre / 1e9,
         "append_prefill_kv_gbs": cnt["prefill_kv_bytes"] / t_pre / 1e6,
-        "decode_kv_append_ms": t_app1, "decode_ms": t_dec,
+        "decode_kv_append_ms": t_app1, "decode_ms": t_dec, "decode_fused_append": True,
         "decode_kv_gbs": (cnt["decode_kv_bytes"] / t_dec / 1e6) if has_decode else None,
     }
     # dominant call of the step and the roofline that bounds it on this workload

@@ -185,6 +185,26 @@ efim_status efim_decode_attn(const efim_cache_desc* cache, int32_t batch,
                              int32_t* d_status, void* stream);
 
 /*
+ * Steps 1 and 3 of a decode step in one launch: the generated token of row s is the row's
+ * last key, position ctx_len[s] - 1.  The kernel rotates its q and k by that position
+ * (the same fp32 arithmetic and single bf16 rounding as efim_kv_append), stores k/v into
+ * the page slot and attends over keys [0, ctx_len[s]) - the result of
+ *     efim_kv_append(cached_len = ctx_len - 1, new_len = 1) ; efim_decode_attn(ctx_len)
+ * bit for bit, with one kernel less per step.  Differences: d_q is read only (the rotated q
+ * is not written back); `rope` may be NULL or hold a NULL table (no rotation); rows with
+ * ctx_len[s] == 0 append nothing.  A position >= rope->max_position sets
+ * EFIM_DEV_BAD_POSITION and skips the row.  d_k_new / d_v_new: [batch][num_kv_heads][head_dim]
+ * bf16.  Workspace and every other argument as for efim_decode_attn.
+ */
+efim_status efim_decode_step(const efim_cache_desc* cache, int32_t batch,
+                             const int32_t* d_ctx_len, int32_t max_ctx_len,
+                             const int32_t* d_block_table, int32_t max_pages_per_seq,
+                             const efim_rope_desc* rope, const void* d_q,
+                             const void* d_k_new, const void* d_v_new, void* d_out, float* d_lse,
+                             float sm_scale, void* d_workspace, size_t workspace_bytes,
+                             int32_t* d_status, void* stream);
+
+/*
  * Allocation-free variant of efim_decode_attn (the paper has no counterpart; this is
  * a convenience of this library).  For callers that cannot provide a workspace
  * because they may not allocate device memory at all - a serving loop that has

@@ -39,7 +39,7 @@ EXPORTS = ("efim_last_cuda_error", "efim_strerror", "efim_version", "efim_rope_t
            "efim_decode_workspace_bytes", "efim_decode_attn",
            "efim_decode_static_scratch_bytes", "efim_decode_attn_static",
            "efim_prefill_launch_count", "efim_decode_launch_count",
-           "efim_prefill_plan_bytes", "efim_prefill_plan", "efim_append_prefill_attn_planned",
+           "efim_prefill_plan_bytes", "efim_prefill_plan", "efim_append_prefill_attn_planned", "efim_decode_step",
            "efim_frontend_create", "efim_frontend_destroy", "efim_frontend_transform", "efim_frontend_admit",
            "efim_frontend_finish", "efim_frontend_stats")
 
@@ -86,6 +86,10 @@ def load_library():
     lib.efim_decode_attn.argtypes = [POINTER(_CacheDesc), c_int32, c_void_p, c_int32, c_void_p, c_int32,
                                      c_void_p, c_void_p, c_void_p, c_float, c_void_p, c_size_t,
                                      c_void_p, c_void_p]
+    lib.efim_decode_step.restype = ctypes.c_int
+    lib.efim_decode_step.argtypes = [POINTER(_CacheDesc), c_int32, c_void_p, c_int32, c_void_p, c_int32,
+                                     POINTER(_RopeDesc), c_void_p, c_void_p, c_void_p, c_void_p, c_void_p, c_float,
+                                     c_void_p, c_size_t, c_void_p, c_void_p]
     lib.efim_prefill_launch_count.restype = c_int32
     lib.efim_prefill_launch_count.argtypes = [POINTER(_CacheDesc), POINTER(_BatchDesc)]
     lib.efim_decode_launch_count.restype = c_int32
@@ -337,3 +341,16 @@ class Frontend:
         out = np.zeros(4, np.int64)
         self._lib.efim_frontend_stats(self._fe, out.ctypes.data)
         return dict(prompt_tokens=int(out[0]), hit_tokens=int(out[1]), evictions=int(out[2]), free_pages=int(out[3]))
+
+
+def efim_decode_step(cache: Cache, batch: int, d_ctx_len, max_ctx_len, d_block_table, rope, q, k_new, v_new, out,
+                     lse=None, sm_scale=0.0, workspace=None, status=None, stream=None):
+    """kv_append of one token per row and decode attention in one launch (q is not modified)."""
+    nbytes = 0 if workspace is None else workspace.numel() * workspace.element_size()
+    st = load_library().efim_decode_step(ctypes.byref(cache.desc), batch, _ptr(d_ctx_len), int(max_ctx_len),
+                                         _ptr(d_block_table), int(d_block_table.shape[1]),
+                                         ctypes.byref(rope.desc) if rope is not None else None,
+                                         _ptr(q), _ptr(k_new), _ptr(v_new), _ptr(out), _ptr(lse), float(sm_scale),
+                                         _ptr(workspace), nbytes, _ptr(status), _stream_ptr(stream))
+    if st != 0:
+        raise EfimError(st, "efim_decode_step")

@@ -63,7 +63,40 @@ __device__ __forceinline__ void dec_bulk_load(uint32_t dst, const void* src, uin
                : "memory");
 }
 
-template <int D, int GT>
+// Rotation of one 16-byte vector (8 bf16) of a head row, exactly as efim_kv_append does it
+// (fp32 FMA, one rounding to bf16).  Rotate-half pairing: `mine` is vector j of the row,
+// `other` vector j ^ (D/16); the first half of the row gets a c - b s, the second b c + a s.
+// Interleaved pairing: the pairs (2f, 2f+1) sit inside the vector and `other` is not used.
+__device__ __forceinline__ uint4 dec_rotate_vec(uint4 mine, uint4 other, const float* cs, int D, int j, int interleaved) {
+  uint32_t* m = reinterpret_cast<uint32_t*>(&mine);
+  const uint32_t* o = reinterpret_cast<const uint32_t*>(&other);
+  if (!interleaved) {
+    const int half = D / 16;
+    const bool first = j < half;
+    const float* c = cs + (j % half) * 8;
+    const float* sn = c + D / 2;
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+      const float m0 = bf16lo(m[i]), m1 = bf16hi(m[i]), o0 = bf16lo(o[i]), o1 = bf16hi(o[i]);
+      const float c0 = __ldg(c + 2 * i), c1 = __ldg(c + 2 * i + 1), s0 = __ldg(sn + 2 * i), s1 = __ldg(sn + 2 * i + 1);
+      const float r0 = first ? fmaf(m0, c0, -(o0 * s0)) : fmaf(m0, c0, o0 * s0);
+      const float r1 = first ? fmaf(m1, c1, -(o1 * s1)) : fmaf(m1, c1, o1 * s1);
+      m[i] = pack_bf16x2(r0, r1);
+    }
+  } else {
+    const float* c = cs + j * 4;
+    const float* sn = c + D / 2;
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+      const float a = bf16lo(m[i]), b = bf16hi(m[i]);
+      const float ci = __ldg(c + i), si = __ldg(sn + i);
+      m[i] = pack_bf16x2(fmaf(a, ci, -(b * si)), fmaf(b, ci, a * si));
+    }
+  }
+  return mine;
+}
+
+template <int D, int GT, bool FUSED>
 __global__ void __launch_bounds__(128, 3) decode_splitkv_kernel(const DecodeParams p) {
   constexpr int LPT = D / 8;            // lanes sharing one token row
   constexpr int TPS = 32 / LPT;         // tokens per warp-wide 16-byte read
@@ -95,6 +128,15 @@ __global__ void __launch_bounds__(128, 3) decode_splitkv_kernel(const DecodePara
   const int begin = c * p.chunk_tokens;
   const int head0 = kvh * G + g0;
   const int tid = threadIdx.x;
+  // fused step: the new token sits at position len - 1; its rotation needs a table row
+  const float* cs_row = nullptr;
+  if (FUSED && len > 0 && p.cos_sin) {
+    if (len - 1 >= p.max_position) {
+      if (tid == 0 && p.status) atomicOr(p.status, EFIM_DEV_BAD_POSITION);
+      return;
+    }
+    cs_row = p.cos_sin + (size_t)(len - 1) * D;
+  }
   if (begin >= len) {
     // nothing visible in this chunk; a row without any key still gets a defined result
     if (len <= 0 && c == 0 && p.n_chunks == 1) {
@@ -151,7 +193,9 @@ __global__ void __launch_bounds__(128, 3) decode_splitkv_kernel(const DecodePara
 #pragma unroll
   for (int g = 0; g < GT; ++g) {
     if (g < ng) {
-      const uint4 w = __ldg(reinterpret_cast<const uint4*>(p.q + ((size_t)r * p.Hq + head0 + g) * D) + j);
+      const uint4* qrow = reinterpret_cast<const uint4*>(p.q + ((size_t)r * p.Hq + head0 + g) * D);
+      uint4 w = __ldg(qrow + j);
+      if (FUSED && cs_row) w = dec_rotate_vec(w, __ldg(qrow + (j ^ (LPT / 2))), cs_row, D, j, p.interleaved);
       const uint32_t* u = reinterpret_cast<const uint32_t*>(&w);
 #pragma unroll
       for (int e = 0; e < 4; ++e) q2[g][e] = pack2(bf16lo(u[e]) * p.scale_log2, bf16hi(u[e]) * p.scale_log2);
@@ -199,6 +243,30 @@ __global__ void __launch_bounds__(128, 3) decode_splitkv_kernel(const DecodePara
         if (lane == 0 && p.status) atomicOr(p.status, EFIM_DEV_TIMEOUT);
         break;
       }
+    }
+    if (FUSED && page_ok && pg == ((len - 1) >> 4)) {
+      // The page of the new token: whatever the copy brought for its slot is replaced, in
+      // shared memory, by the token's rotated k and its v; the CTA of the kv head's first
+      // group tile also puts them into the pools.  (Other CTAs that read this page patch
+      // their own copy the same way, so nobody depends on when the pool is written.)
+      if (tg == 0) {
+        const int slot = (len - 1) & 15;
+        const uint4* krow = reinterpret_cast<const uint4*>(p.k_new + ((size_t)r * p.Hkv + kvh) * D);
+        const uint4* vrow = reinterpret_cast<const uint4*>(p.v_new + ((size_t)r * p.Hkv + kvh) * D);
+        uint4 kv = __ldg(krow + j);
+        if (cs_row) kv = dec_rotate_vec(kv, __ldg(krow + (j ^ (LPT / 2))), cs_row, D, j, p.interleaved);
+        const uint4 vv = __ldg(vrow + j);
+        uint8_t* kpage = ring + sg * 2 * PAGE_BYTES;
+        *reinterpret_cast<uint4*>(kpage + (slot * D + j * 8) * 2) = kv;
+        *reinterpret_cast<uint4*>(kpage + PAGE_BYTES + (slot * D + j * 8) * 2) = vv;
+        if (g0 == 0) {
+          const int pid = __ldg(bt + pg);
+          const size_t off = (((size_t)pid * p.Hkv + kvh) * 16 + slot) * D + j * 8;
+          *reinterpret_cast<uint4*>(p.k_pool_w + off) = kv;
+          *reinterpret_cast<uint4*>(p.v_pool_w + off) = vv;
+        }
+      }
+      __syncwarp();
     }
     if (page_ok) {
       const uint8_t* kst = ring + sg * 2 * PAGE_BYTES + (tg * D + j * 8) * 2;
@@ -407,13 +475,17 @@ DecodePlan plan_decode(int rows, int Hq, int Hkv, int D, int max_len) {
   return pl;
 }
 
+template <int D, int GT, bool FUSED>
+static efim_status launch_split_f(const DecodeParams& p, dim3 grid, cudaStream_t s) {
+  constexpr int ring_bytes = 4 * DEC_STAGES * 2 * 16 * D * 2;      // 4 warps x stages x (K page + V page)
+  EFIM_CUDA_TRY(cudaFuncSetAttribute(decode_splitkv_kernel<D, GT, FUSED>,
+                                     cudaFuncAttributeMaxDynamicSharedMemorySize, ring_bytes));
+  decode_splitkv_kernel<D, GT, FUSED><<<grid, 128, ring_bytes, s>>>(p);
+  return EFIM_OK;
+}
 template <int D, int GT>
 static efim_status launch_split(const DecodeParams& p, dim3 grid, cudaStream_t s) {
-  constexpr int ring_bytes = 4 * DEC_STAGES * 2 * 16 * D * 2;      // 4 warps x stages x (K page + V page)
-  EFIM_CUDA_TRY(cudaFuncSetAttribute(decode_splitkv_kernel<D, GT>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                     ring_bytes));
-  decode_splitkv_kernel<D, GT><<<grid, 128, ring_bytes, s>>>(p);
-  return EFIM_OK;
+  return p.fused ? launch_split_f<D, GT, true>(p, grid, s) : launch_split_f<D, GT, false>(p, grid, s);
 }
 
 template <int D>
@@ -458,11 +530,12 @@ extern "C" int32_t efim_decode_launch_count(const efim_cache_desc* cache, int32_
   return pl.n_chunks > 1 ? 2 : 1;
 }
 
-extern "C" efim_status efim_decode_attn(const efim_cache_desc* cache, int32_t batch, const int32_t* d_ctx_len,
-                                        int32_t max_ctx_len, const int32_t* d_block_table,
-                                        int32_t max_pages_per_seq, const void* d_q, void* d_out, float* d_lse,
-                                        float sm_scale, void* d_workspace, size_t workspace_bytes,
-                                        int32_t* d_status, void* stream) {
+// efim_decode_attn, and efim_decode_step when d_k_new / d_v_new are given
+static efim_status decode_entry(const efim_cache_desc* cache, int32_t batch, const int32_t* d_ctx_len,
+                                int32_t max_ctx_len, const int32_t* d_block_table, int32_t max_pages_per_seq,
+                                const efim_rope_desc* rope, const void* d_k_new, const void* d_v_new, bool fused,
+                                const void* d_q, void* d_out, float* d_lse, float sm_scale, void* d_workspace,
+                                size_t workspace_bytes, int32_t* d_status, void* stream) {
   efim_status st = efim::check_cache(cache);
   if (st != EFIM_OK) return st;
   if (batch < 0 || max_pages_per_seq <= 0) return EFIM_ERR_INVALID_ARG;
@@ -500,5 +573,39 @@ extern "C" efim_status efim_decode_attn(const efim_cache_desc* cache, int32_t ba
   p.n_chunks = pl.n_chunks;
   const float scale = sm_scale > 0.f ? sm_scale : 1.0f / sqrtf((float)cache->head_dim);
   p.scale_log2 = scale * 1.4426950408889634f;
+  if (fused) {
+    if (!d_k_new || !d_v_new) return EFIM_ERR_INVALID_ARG;
+    if ((reinterpret_cast<uintptr_t>(d_k_new) | reinterpret_cast<uintptr_t>(d_v_new)) & 15) return EFIM_ERR_INVALID_ARG;
+    p.fused = 1;
+    p.k_new = static_cast<const uint16_t*>(d_k_new);
+    p.v_new = static_cast<const uint16_t*>(d_v_new);
+    p.k_pool_w = static_cast<uint16_t*>(cache->d_k_pool);
+    p.v_pool_w = static_cast<uint16_t*>(cache->d_v_pool);
+    if (rope && rope->d_cos_sin) {
+      if (rope->max_position <= 0 || (reinterpret_cast<uintptr_t>(rope->d_cos_sin) & 15)) return EFIM_ERR_INVALID_ARG;
+      p.cos_sin = rope->d_cos_sin;
+      p.max_position = rope->max_position;
+      p.interleaved = rope->interleaved;
+    }
+  }
   return efim::launch_decode(p, pl, cache->head_dim, static_cast<cudaStream_t>(stream));
+}
+
+extern "C" efim_status efim_decode_attn(const efim_cache_desc* cache, int32_t batch, const int32_t* d_ctx_len,
+                                        int32_t max_ctx_len, const int32_t* d_block_table,
+                                        int32_t max_pages_per_seq, const void* d_q, void* d_out, float* d_lse,
+                                        float sm_scale, void* d_workspace, size_t workspace_bytes,
+                                        int32_t* d_status, void* stream) {
+  return decode_entry(cache, batch, d_ctx_len, max_ctx_len, d_block_table, max_pages_per_seq, nullptr, nullptr,
+                      nullptr, false, d_q, d_out, d_lse, sm_scale, d_workspace, workspace_bytes, d_status, stream);
+}
+
+extern "C" efim_status efim_decode_step(const efim_cache_desc* cache, int32_t batch, const int32_t* d_ctx_len,
+                                        int32_t max_ctx_len, const int32_t* d_block_table,
+                                        int32_t max_pages_per_seq, const efim_rope_desc* rope, const void* d_q,
+                                        const void* d_k_new, const void* d_v_new, void* d_out, float* d_lse,
+                                        float sm_scale, void* d_workspace, size_t workspace_bytes,
+                                        int32_t* d_status, void* stream) {
+  return decode_entry(cache, batch, d_ctx_len, max_ctx_len, d_block_table, max_pages_per_seq, rope, d_k_new,
+                      d_v_new, true, d_q, d_out, d_lse, sm_scale, d_workspace, workspace_bytes, d_status, stream);
 }

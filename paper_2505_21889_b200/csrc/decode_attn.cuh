@@ -19,6 +19,15 @@ struct DecodeParams {
   int32_t* status;
   int R, Hq, Hkv, max_pages_per_seq, num_pages, chunk_tokens, n_chunks;
   float scale_log2;           // sm_scale * log2(e)
+  // fused decode step: the row's last key (position row_len[r] - 1) is this step's new token.
+  // Its k/v are rotated, put into the page slot and used from shared memory in the same
+  // kernel; q comes in unrotated.  All null / 0 for a plain decode.
+  const uint16_t* k_new;      // [R][Hkv][D]
+  const uint16_t* v_new;
+  uint16_t* k_pool_w;         // the pools again, writable
+  uint16_t* v_pool_w;
+  const float* cos_sin;       // [max_position][D] or null (no rotation)
+  int fused, interleaved, max_position;
 };
 
 struct DecodePlan {

@@ -9,7 +9,7 @@ under three schemes -
 Every round batches the users' requests: the front end (efim_frontend_*) turns each request
 into a prompt, a cached length and a block-table row; the tokens that are not cached go
 through efim_kv_append + efim_append_prefill_attn, the generated tokens through
-efim_kv_append + efim_decode_attn, one step per token.  A pool smaller than the users'
+efim_decode_step (append fused with decode attention), one step per token.  A pool smaller than the users'
 working set makes the front end evict and the reuse rate fall (Sec. 5.3, sensitivity to
 the number of users).  Only the attention path of ONE layer is timed - no linear layers,
 no sampling - so the ratios are those of this path, not of end-to-end serving.
@@ -117,15 +117,12 @@ def run_scheme(scheme, sessions, layer, pool_pages, max_pages_per_seq, observe=N
         gen_ids = np.array([[sessions[g][r]["gen"][s] for g in group] for s in range(steps)]).reshape(-1)
         dq_all, dk_all, dv_all = (x.view(steps, users, *x.shape[1:]) for x in layer.qkv(gen_ids))
         dec_all = torch.empty_like(dq_all)
-        step_batches = [efim.Batch(ctx + s, one, d_bt, layer.device) for s in range(steps)]
         d_ctx_all = torch.from_numpy(np.stack([ctx + s + 1 for s in range(steps)])).to(layer.device)
 
         def decode_loop():
             for s in range(steps):
-                efim.efim_kv_append(layer.cache, step_batches[s], layer.rope, dq_all[s], dk_all[s], dv_all[s],
-                                    layer.status)
-                efim.efim_decode_attn(layer.cache, users, d_ctx_all[s], max_ctx, d_bt, dq_all[s], dec_all[s], None,
-                                      0.0, dws, layer.status)
+                efim.efim_decode_step(layer.cache, users, d_ctx_all[s], max_ctx, d_bt, layer.rope, dq_all[s],
+                                      dk_all[s], dv_all[s], dec_all[s], None, 0.0, dws, layer.status)
         if graph and steps > 0:
             g = torch.cuda.CUDAGraph()
             torch.cuda.synchronize()

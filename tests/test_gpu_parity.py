@@ -274,3 +274,45 @@ def test_planned_prefill_is_bit_identical_and_checks_its_plan(name):
     assert e.value.code == 1
     with pytest.raises(efim.EfimError):                    # a truncated blob
         efim.efim_append_prefill_attn(dw.cache, dw.batch, dw.q, dw.out, dw.lse, 0.0, dw.ws, dw.status, plan=plan[:64])
+
+
+@pytest.mark.parametrize("Hq,Hkv,D,interleaved,use_rope", [
+    (8, 2, 128, False, True),     # group of 4: one CTA per kv head
+    (7, 1, 128, False, True),     # group of 7: two CTAs share the new token's page
+    (4, 4, 64, True, True),       # head_dim 64, interleaved pairing
+    (6, 2, 64, False, False),     # no rotation
+])
+def test_fused_decode_step_equals_append_then_decode(Hq, Hkv, D, interleaved, use_rope):
+    """efim_decode_step against efim_kv_append + efim_decode_attn on the same inputs, over
+    several steps (page edges included): outputs, lse and the pools bit for bit; q untouched."""
+    H = _harness()
+    import paper_2505_21889_b200 as efim
+    ctx0 = [15, 16, 31, 300, 1, 700]
+    w = _custom(Hq, Hkv, D, ctx0, [0] * len(ctx0), seed=11, extra=6)
+    a, b = H.DeviceWorkload(w, interleaved=interleaved, use_rope=use_rope), \
+        H.DeviceWorkload(w, interleaved=interleaved, use_rope=use_rope)
+    B = w.batch
+    ctx = np.array(ctx0, np.int32)
+    max_ctx = int(ctx.max()) + 6
+    ws_a = torch.empty(max(efim.efim_decode_workspace_bytes(a.cache, B, max_ctx), 256), dtype=torch.uint8, device="cuda")
+    ws_b = torch.empty_like(ws_a)
+    one = np.ones(B, np.int32)
+    for step in range(6):
+        q, k, v = w.decode_qkv(step)
+        qa, ka, va = H.bits_to_torch(q), H.bits_to_torch(k), H.bits_to_torch(v)
+        qb, kb, vb = qa.clone(), ka.clone(), va.clone()
+        d_ctx = torch.from_numpy(ctx + 1).cuda()
+        out_a, out_b = torch.empty_like(qa), torch.empty_like(qa)
+        lse_a = torch.empty((B, Hq), dtype=torch.float32, device="cuda")
+        lse_b = torch.empty_like(lse_a)
+        efim.efim_kv_append(a.cache, efim.Batch(ctx, one, a.batch.d_block_table), a.rope, qa, ka, va, a.status)
+        efim.efim_decode_attn(a.cache, B, d_ctx, max_ctx, a.batch.d_block_table, qa, out_a, lse_a, 0.0, ws_a, a.status)
+        efim.efim_decode_step(b.cache, B, d_ctx, max_ctx, b.batch.d_block_table, b.rope, qb, kb, vb, out_b, lse_b, 0.0,
+                              ws_b, b.status)
+        torch.cuda.synchronize()
+        assert int(a.status.item()) == 0 and int(b.status.item()) == 0
+        assert torch.equal(out_a.view(torch.int16), out_b.view(torch.int16)) and torch.equal(lse_a, lse_b), step
+        assert torch.equal(qb.view(torch.int16), H.bits_to_torch(q).view(torch.int16))      # q is read only
+        ctx = ctx + 1
+    assert torch.equal(a.k_pool.view(torch.int16), b.k_pool.view(torch.int16))
+    assert torch.equal(a.v_pool.view(torch.int16), b.v_pool.view(torch.int16))
