@@ -451,7 +451,7 @@ def run_native(args):
             roof = {"kernel": "efim_append_prefill_attn", "bound": "hbm",
                     "achieved": breakdown["append_prefill_kv_gbs"], "peak": peaks["hbm_gbs"], "unit": "GB/s"}
     else:
-        roof = {"kernel": "efim_decode_attn", "bound": "hbm", "achieved": breakdown["decode_kv_gbs"],
+        roof = {"kernel": "efim_decode_step", "bound": "hbm", "achieved": breakdown["decode_kv_gbs"],
                 "peak": peaks["hbm_gbs"], "unit": "GB/s"}
     roof["frac"] = roof["achieved"] / roof["peak"]
     roof["peak_source"] = peaks["source"]
