@@ -97,6 +97,14 @@ def test_cfg5_full_decode_steps_sampled():
         H.assert_attn_close(H.torch_to_bits(out)[seqs], o, f"cfg5 full decode step {step}")
         assert np.abs(lse_d.cpu().numpy()[seqs] - lse).max() <= H.LSE_TOL
         assert torch.isfinite(out.float()).all()
+        # the fused step on the same inputs (it stores the same k/v again): identical bits at full size
+        out_f = torch.empty_like(out)
+        lse_f = torch.empty_like(lse_d)
+        efim.efim_decode_step(dw.cache, B, torch.from_numpy(ctx_all).cuda(), max_ctx, dw.batch.d_block_table, dw.rope,
+                              H.bits_to_torch(q), dk, dv, out_f, lse_f, 0.0, ws, dw.status)
+        torch.cuda.synchronize()
+        assert int(dw.status.item()) == 0
+        assert torch.equal(out_f.view(torch.int16), out.view(torch.int16)) and torch.equal(lse_f, lse_d)
     for r, s in enumerate(seqs):
         pg = w.pages_of(s, int(ctx_all[s]))[-2:]
         want = vp[bt[r, len(w.pages_of(s, int(ctx_all[s]))) - 2: len(w.pages_of(s, int(ctx_all[s])))]]
