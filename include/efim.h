@@ -292,6 +292,23 @@ efim_status efim_frontend_finish(efim_frontend* fe, int64_t handle, const int32_
 /* h_out[0..4) = prompt tokens admitted, of which found cached, pages evicted, pages free now. */
 void efim_frontend_stats(const efim_frontend* fe, int64_t* h_out);
 
+/* ------------------------------------------------------------------------------------
+ * Fragment tokenisation, Sec. 3.2 (Fig. 8: "the length of each segment follows uniform
+ * distribution [1,200]"): the training-side data processing that teaches a model to emit
+ * sub-word pieces anywhere.  The library decides where a text is cut; the caller
+ * tokenises every segment on its own and concatenates the ids.  Host only.
+ * Lengths count characters (the paper does not say) and are lo + z_i mod (hi - lo + 1)
+ * with z_i the i-th draw of SplitMix64 under `seed`; the last segment is what is left.
+ *
+ * efim_fragment_cuts: writes the end offsets of the segments of a text of n characters
+ * (the last one is n) into h_cuts, at most `capacity` of them, and returns how many there
+ * are (so call with capacity 0 to size); -1 for invalid arguments (n < 0, lo < 1, hi < lo).
+ * efim_fim_split: the two cut points 0 <= a <= b <= n of the FIM transformation of a
+ * document (prefix [0,a), middle [a,b), suffix [b,n); Sec. 2.1), both uniform on [0, n].
+ */
+int64_t efim_fragment_cuts(uint64_t seed, int64_t n, int32_t lo, int32_t hi, int64_t* h_cuts, int64_t capacity);
+efim_status efim_fim_split(uint64_t seed, int64_t n, int64_t* a, int64_t* b);
+
 #ifdef __cplusplus
 }
 #endif
