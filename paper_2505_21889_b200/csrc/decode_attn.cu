@@ -436,16 +436,40 @@ __global__ void __launch_bounds__(128) decode_merge_kernel(const DecodeParams p)
   const int nc = (len + p.chunk_tokens - 1) / p.chunk_tokens;
   const float* pl = p.part_lse + row_head * p.n_chunks;
   const float* po = p.part_o + row_head * p.n_chunks * D + lane * EPL;
+  // the lanes fetch the chunks' lse values side by side; the partial rows are then loaded four
+  // at a time and folded in chunk order (a chain of dependent loads cost more than the split
+  // kernel's tail on short steps)
   float M = -INFINITY;
-  for (int c = 0; c < nc; ++c) M = fmaxf(M, pl[c]);
+  for (int c0 = 0; c0 < nc; c0 += 32)
+    if (c0 + lane < nc) M = fmaxf(M, __ldg(pl + c0 + lane));
+#pragma unroll
+  for (int d = 16; d > 0; d >>= 1) M = fmaxf(M, __shfl_xor_sync(0xffffffffu, M, d));
   float L = 0.f, acc[EPL];
 #pragma unroll
   for (int e = 0; e < EPL; ++e) acc[e] = 0.f;
-  for (int c = 0; c < nc; ++c) {
-    const float w = exp2f(pl[c] - M);
-    L += w;
+  for (int c0 = 0; c0 < nc; c0 += 4) {
+    float w[4];
+    __align__(16) float v[4][EPL];
 #pragma unroll
-    for (int e = 0; e < EPL; ++e) acc[e] = fmaf(w, po[(size_t)c * D + e], acc[e]);
+    for (int i = 0; i < 4; ++i) {
+      if (c0 + i < nc) {
+        w[i] = __ldg(pl + c0 + i);
+        if constexpr (EPL == 4) {
+          *reinterpret_cast<float4*>(v[i]) = __ldg(reinterpret_cast<const float4*>(po + (size_t)(c0 + i) * D));
+        } else {
+          *reinterpret_cast<float2*>(v[i]) = __ldg(reinterpret_cast<const float2*>(po + (size_t)(c0 + i) * D));
+        }
+      }
+    }
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+      if (c0 + i < nc) {
+        const float wi = exp2f(w[i] - M);
+        L += wi;
+#pragma unroll
+        for (int e = 0; e < EPL; ++e) acc[e] = fmaf(wi, v[i][e], acc[e]);
+      }
+    }
   }
   const float inv = 1.f / L;
 #pragma unroll
