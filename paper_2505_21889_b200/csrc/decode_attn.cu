@@ -121,6 +121,14 @@ __global__ void __launch_bounds__(128, 3) decode_splitkv_kernel(const DecodePara
   const int g0 = (blockIdx.y % gsplit) * GT;
   const int ng = min(GT, G - g0);
   const int c = blockIdx.z;
+  // The first block-table entries of every warp are fetched before the row's length is known
+  // (any entry of the row may be read; those past the length are dropped below), so that the
+  // two loads share one round trip: a short step's time is mostly this ramp.
+  const int seq = p.row_seq ? __ldg(p.row_seq + r) : r;
+  const int32_t* bt = p.block_table + (size_t)seq * p.max_pages_per_seq;
+  const int first_pg = ((c * p.chunk_tokens) >> 4) + (threadIdx.x >> 5);
+  const int my_pg = first_pg + 4 * (threadIdx.x & 31);
+  const int pid_early = my_pg < p.max_pages_per_seq ? __ldg(bt + my_pg) : -1;
   int len = __ldg(p.row_len + r);
   if (len > p.max_pages_per_seq * 16) {           // longer than the block table can address: clamp and report
     len = p.max_pages_per_seq * 16;
@@ -147,13 +155,10 @@ __global__ void __launch_bounds__(128, 3) decode_splitkv_kernel(const DecodePara
     return;
   }
   const int end = min(len, begin + p.chunk_tokens);
-  const int seq = p.row_seq ? __ldg(p.row_seq + r) : r;
   const int lane = tid & 31, warp = tid >> 5;
   const int j = lane % LPT, tg = lane / LPT;
 
   // ---- this warp's pages: first_pg, first_pg + 4, ... ; start their copies before anything else
-  const int32_t* bt = p.block_table + (size_t)seq * p.max_pages_per_seq;
-  const int first_pg = (begin >> 4) + warp;
   const int last_pg = (end - 1) >> 4;
   const int n_pages = first_pg <= last_pg ? (last_pg - first_pg) / 4 + 1 : 0;
   uint8_t* ring = dec_ring + warp * (DEC_STAGES * 2 * PAGE_BYTES);
@@ -164,7 +169,7 @@ __global__ void __launch_bounds__(128, 3) decode_splitkv_kernel(const DecodePara
   }
   __syncwarp();
   // page ids of the next 32 pages of this warp, one per lane (refilled every 32 pages)
-  int pid_cache = (lane < n_pages) ? __ldg(bt + first_pg + 4 * lane) : -1;
+  int pid_cache = (lane < n_pages) ? pid_early : -1;
   auto issue = [&](int i) {             // start the copies of this warp's i-th page into stage i % DEC_STAGES
     const int pid = __shfl_sync(0xffffffffu, pid_cache, i & 31);
     const bool ok = pid >= 0 && pid < p.num_pages;
