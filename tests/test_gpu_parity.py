@@ -160,6 +160,38 @@ def test_decode_loop_small(name):
         assert np.abs(lse_d.cpu().numpy() - lse).max() <= H.LSE_TOL
 
 
+def test_decode_one_long_row_many_chunks():
+    """A lone long row is cut into more than 32 chunks (so that every SM gets work); the merge
+    then takes more than one pass over the lanes for the chunks' lse values."""
+    H = _harness()
+    import paper_2505_21889_b200 as efim
+    Hq, Hkv, D = 8, 2, 128
+    w = _custom(Hq, Hkv, D, [12000, 40], [0, 0], seed=5, extra=2)
+    dw = H.DeviceWorkload(w)
+    kp, vp, bt, seqs = w.compact_host_pool()
+    ctx = w.cached_len.astype(np.int32).copy()
+    B = w.batch
+    max_ctx = int(ctx.max()) + 2
+    nbytes = efim.efim_decode_workspace_bytes(dw.cache, B, max_ctx)
+    assert nbytes > 33 * B * Hq * D * 4, "expected more than 32 chunks"
+    ws = torch.empty(nbytes, dtype=torch.uint8, device="cuda")
+    one = np.ones(B, np.int32)
+    for step in range(2):
+        q, k, v = w.decode_qkv(step)
+        q_rot = orc.kv_append(kp, vp, bt, ctx, one, q, k, v, w.rope_base)
+        ctx = ctx + 1
+        o, lse = orc.decode_attention(q_rot, kp, vp, bt, ctx, Hq)
+        dq, dk, dv = H.bits_to_torch(q), H.bits_to_torch(k), H.bits_to_torch(v)
+        out = torch.empty_like(dq)
+        lse_d = torch.empty((B, Hq), dtype=torch.float32, device="cuda")
+        efim.efim_decode_step(dw.cache, B, torch.from_numpy(ctx).cuda(), max_ctx, dw.batch.d_block_table, dw.rope,
+                              dq, dk, dv, out, lse_d, 0.0, ws, dw.status)
+        torch.cuda.synchronize()
+        assert int(dw.status.item()) == 0
+        H.assert_attn_close(H.torch_to_bits(out), o, f"long row, step {step}")
+        assert np.abs(lse_d.cpu().numpy() - lse).max() <= H.LSE_TOL
+
+
 def test_decode_zero_length_and_bad_page_flag():
     H = _harness()
     import paper_2505_21889_b200 as efim
