@@ -68,13 +68,21 @@ __global__ void __launch_bounds__(KV_APPEND_THREADS) kv_append_kernel(const KvAp
   const int lane = threadIdx.x % LANES;
   const int t = blockIdx.x * (KV_APPEND_THREADS / LANES) + threadIdx.x / LANES;
   if (t >= p.total_new_tokens) return;
-  // sequence of this token: last s with q_indptr[s] <= t
-  int lo = 0, hi = p.batch;
-  while (hi - lo > 1) {
-    int mid = (lo + hi) >> 1;
-    if (__ldg(p.q_indptr + mid) <= t) lo = mid; else hi = mid;
+  // sequence of this token: last s with q_indptr[s] <= t.  Up to 32 sequences are probed by the
+  // warp's lanes at once (one round trip instead of a chain of five); more by bisection.
+  int s;
+  if (p.batch <= 32) {
+    const int wl = threadIdx.x & 31;
+    const bool le = wl < p.batch && __ldg(p.q_indptr + wl) <= t;
+    s = 31 - __clz((int)(__ballot_sync(0xffffffffu, le) | 1u));
+  } else {
+    int lo = 0, hi = p.batch;
+    while (hi - lo > 1) {
+      int mid = (lo + hi) >> 1;
+      if (__ldg(p.q_indptr + mid) <= t) lo = mid; else hi = mid;
+    }
+    s = lo;
   }
-  const int s = lo;
   const int pos = __ldg(p.cached_len + s) + (t - __ldg(p.q_indptr + s));
   const int page_idx = pos >> 4;
   int err = 0;
