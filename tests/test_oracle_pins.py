@@ -372,6 +372,64 @@ def test_hand_derived_golden_example():
     assert abs(lse[0, 0] - vals["lse"][0]) < 1e-6
 
 
+# ---------------------------------------------------------------- kv_append's position rule
+def test_kv_append_from_an_empty_cache_starts_at_position_zero():
+    """Sec. 1: `inc` follows `<P>prefix<S>suffix<M>`, so a token's position is its
+    index in the reordered prompt and the first token of an empty cache has
+    position 0 - where the rotation is the identity.  Token 0 must come back
+    bit for bit and land in page block_table[s][0], slot 0; token 1 must not
+    (it is turned by one radian on the fastest pair)."""
+    rng = np.random.default_rng(30)
+    B, Hq, Hkv, D, P = 2, 2, 2, 8, 16
+    new = np.array([3, 18], np.int32)
+    k_pool, v_pool, bt, cached, new, q, k, v = _random_paged_case(rng, B, Hq, Hkv, D, P, [0, 0], new)
+    k_before = k_pool.copy()
+    q_rot = orc.kv_append(k_pool, v_pool, bt, cached, new, q, k, v, 10000.0)
+    t = 0
+    for s in range(B):
+        assert np.array_equal(q_rot[t], q[t])
+        assert np.array_equal(k_pool[bt[s, 0], :, 0, :], k[t])
+        assert np.array_equal(v_pool[bt[s, 0], :, 0, :], v[t])
+        assert not np.array_equal(q_rot[t + 1], q[t + 1])
+        assert not np.array_equal(k_pool[bt[s, 0], :, 1, :], k[t + 1])
+        t += int(new[s])
+    # the 18-token sequence spills into its second page at slots 0 and 1 only
+    assert np.array_equal(k_pool[bt[1, 1], :, 2:, :], k_before[bt[1, 1], :, 2:, :])
+    assert not np.array_equal(k_pool[bt[1, 1], :, :2, :], k_before[bt[1, 1], :, :2, :])
+
+
+def test_kv_append_turns_token_i_by_cached_len_plus_i_radians():
+    """D = 2 has the single frequency theta_0 = 1, so new token i of a sequence
+    with C cached tokens is the input times e^{i(C+i)} as a complex number
+    (computed here with cmath, not with the oracle's formula), rounded once to
+    bf16.  An offset of one position turns by one more radian: far outside the
+    rounding."""
+    import cmath
+    rng = np.random.default_rng(31)
+    B, Hq, Hkv, D, P = 2, 3, 1, 2, 16
+    C = np.array([37, 5], np.int32)
+    N = np.array([4, 13], np.int32)
+    k_pool, v_pool, bt, C, N, q, k, v = _random_paged_case(rng, B, Hq, Hkv, D, P, C, N)
+    q_rot = orc.kv_append(k_pool, v_pool, bt, C, N, q, k, v, 777.0)
+    qf, kf = bf16_bits_to_f32(q).astype(np.float64), bf16_bits_to_f32(k).astype(np.float64)
+    t = 0
+    for s in range(B):
+        for i in range(int(N[s])):
+            pos = int(C[s]) + i
+            turn = cmath.exp(1j * pos)
+            for h in range(Hq):
+                z = complex(qf[t, h, 0], qf[t, h, 1]) * turn
+                got = bf16_bits_to_f32(q_rot[t, h]).astype(np.float64)
+                assert abs(got[0] - z.real) <= 2.0 ** -8 * abs(z.real) + 1e-30
+                assert abs(got[1] - z.imag) <= 2.0 ** -8 * abs(z.imag) + 1e-30
+            z = complex(kf[t, 0, 0], kf[t, 0, 1]) * turn
+            got = bf16_bits_to_f32(k_pool[bt[s, pos // P], 0, pos % P]).astype(np.float64)
+            assert abs(got[0] - z.real) <= 2.0 ** -8 * abs(z.real) + 1e-30
+            assert abs(got[1] - z.imag) <= 2.0 ** -8 * abs(z.imag) + 1e-30
+            assert np.array_equal(v_pool[bt[s, pos // P], 0, pos % P], v[t, 0])
+            t += 1
+
+
 # ---------------------------------------------------------------- the paper's invariants
 def _full_turn(rng, B, Hq, Hkv, D, cached, new, base=10000.0, interleaved=False):
     P = 16
@@ -485,7 +543,7 @@ def test_decode_is_append_with_one_token():
 
 
 # ---------------------------------------------------------------- planted mistakes are caught
-@pytest.mark.parametrize("mistake", ["sin_sign", "mask_off_by_one", "gqa_map", "no_scale"])
+@pytest.mark.parametrize("mistake", ["sin_sign", "mask_off_by_one", "gqa_map", "no_scale", "position_off_by_one"])
 def test_pins_catch_planted_mistakes(mistake, monkeypatch):
     """Plant a plausible bug in the oracle (CPU only) and check a pin fails."""
     if mistake == "sin_sign":
@@ -494,6 +552,15 @@ def test_pins_catch_planted_mistakes(mistake, monkeypatch):
         with pytest.raises(AssertionError):
             test_rope_d2_is_plane_rotation_by_p_radians()
         monkeypatch.undo()
+    elif mistake == "position_off_by_one":
+        src = orc.rope_rotate
+        def broken(x_bits, positions, base, interleaved=False):               # pos = C + i + 1
+            return src(x_bits, np.asarray(positions) + 1, base, interleaved)
+        monkeypatch.setattr(orc, "rope_rotate", broken)
+        with pytest.raises(AssertionError):
+            test_kv_append_from_an_empty_cache_starts_at_position_zero()
+        with pytest.raises(AssertionError):
+            test_kv_append_turns_token_i_by_cached_len_plus_i_radians()
     elif mistake == "mask_off_by_one":
         src = orc.append_prefill_attention
         def broken(q, kp, vp, bt, c, n, hq, sm_scale=None):
