@@ -15,10 +15,19 @@
  *
  * Conventions for every entry point
  *   - Pointers named d_* are DEVICE pointers, h_* are HOST pointers.  The caller
- *     owns all memory and the stream; the library allocates no device memory and,
- *     apart from the fixed array of efim_decode_attn_static, keeps no state between calls; it never synchronises the device.
+ *     owns all memory and the stream; the library allocates no device memory and never
+ *     synchronises the device.  What it keeps between calls: the fixed array of
+ *     efim_decode_attn_static (and its per-device address), the SM count of each device it
+ *     has planned for, and the driver entry point it encodes tensor maps with - host-side
+ *     look-ups made once; no call's result depends on an earlier call.
  *   - `stream` is a cudaStream_t passed as void* (NULL = default stream).  All
  *     work is enqueued on it; results are ready when the stream reaches that point.
+ *   - Stream capture: calls that copy a work list from pageable host memory must not be
+ *     issued while the stream is capturing - efim_append_prefill_attn, and
+ *     efim_append_prefill_step without a plan.  The planned calls can be captured with
+ *     lists_resident = 1 (they only launch), or with lists_resident = 0 and a blob in pinned
+ *     memory that outlives the graph.  efim_kv_append, efim_decode_attn and efim_decode_step
+ *     only launch.
  *   - bf16 tensors are raw 16-bit patterns.  Packed layouts, innermost last:
  *       q / out      [total_new_tokens][num_q_heads][head_dim]   bf16
  *       k_new/v_new  [total_new_tokens][num_kv_heads][head_dim]  bf16
@@ -100,7 +109,10 @@ typedef struct {
 } efim_rope_desc;
 
 /* Fill a HOST table for efim_rope_desc (computed in double, rounded to float).
- * h_out: [max_position][head_dim] floats owned by the caller. */
+ * h_out: [max_position][head_dim] floats owned by the caller.  The paper fixes only the
+ * token order (Sec. 1), hence each token's position; the rotary embedding itself is that of
+ * the model families it serves (Sec. 4.1), read here as theta_f = base^(-2f/head_dim), no
+ * scaling. */
 efim_status efim_rope_table_build(double base, int32_t head_dim, int32_t max_position, float* h_out);
 
 /*
@@ -121,6 +133,9 @@ efim_status efim_kv_append(const efim_cache_desc* cache, const efim_batch_desc* 
  * Step 2 (EFIM Sec. 1, Sec. 2.2: prefix and suffix KV are cache hits, so the
  * prefill that remains is the `inc` tokens attending over everything before
  * them).  The new tokens' k/v must already be in the pages (efim_kv_append).
+ * A block-table entry outside [0, num_pages) among the pages a row sees sets
+ * EFIM_DEV_BAD_PAGE; the 16 keys of that page are taken as zeros (the rows that see it are
+ * finite and meaningless, all other rows unaffected).
  * New token i of sequence s (position C+i) sees keys j <= C+i:
  *   out[t,h,:] = sum_j softmax_j(sm_scale * q[t,h,:].k[j,h/G,:]) v[j,h/G,:]
  *   lse[t,h]   = log sum_j exp(sm_scale * q.k_j)         (natural log; optional)
@@ -162,6 +177,30 @@ efim_status efim_append_prefill_attn_planned(const efim_cache_desc* cache, const
                                              int32_t* d_status, void* stream);
 
 /*
+ * Steps 1 and 2 of a turn in one call (EFIM Sec. 1: the `inc` tokens join the cache after
+ * `<P>prefix<S>suffix<M>` and attend over everything before them).  Equivalent to
+ *     efim_kv_append(rope, d_q, d_k_new, d_v_new) ; efim_append_prefill_attn[_planned](d_q)
+ * - out, lse and the pools bit for bit - but d_q is READ ONLY: the attention kernel rotates
+ * each query row by its position cached_len[s] + i as it loads it (the same fp32 arithmetic
+ * and single bf16 rounding), and the append moves only k and v.  The rotated q is never
+ * written, which at equal head counts is two thirds of what efim_kv_append moves.
+ * h_plan = NULL: the work list is planned inside the call (as efim_append_prefill_attn does);
+ * otherwise h_plan / plan_bytes / lists_resident are those of
+ * efim_append_prefill_attn_planned.  `rope` may be NULL or hold a NULL table (no rotation).
+ * A query position >= rope->max_position sets EFIM_DEV_BAD_POSITION; that row attends with a
+ * zero query (its output is finite and meaningless), its k/v are not appended.
+ * d_k_new and d_v_new may both be NULL: the new tokens' k/v are then taken to be in the
+ * pages already (an earlier efim_kv_append with d_q = NULL) and only the attention runs.
+ * Two kernels are enqueued (three when the key range is split).
+ */
+efim_status efim_append_prefill_step(const efim_cache_desc* cache, const efim_batch_desc* batch,
+                                     const efim_rope_desc* rope, const void* d_q,
+                                     const void* d_k_new, const void* d_v_new, void* d_out, float* d_lse,
+                                     float sm_scale, const void* h_plan, size_t plan_bytes,
+                                     int32_t lists_resident, void* d_workspace, size_t workspace_bytes,
+                                     int32_t* d_status, void* stream);
+
+/*
  * Step 3 (decode of the generated middle, EFIM Sec. 2.2 / Fig. 4): one query
  * token per sequence over keys [0, ctx_len[s]) (ctx_len counts the token just
  * appended).  The key range is cut into fixed-length chunks; each chunk yields a
@@ -169,7 +208,10 @@ efim_status efim_append_prefill_attn_planned(const efim_cache_desc* cache, const
  *   lse = log sum_c exp(lse_c),  o = sum_c exp(lse_c - lse) o_c.
  * max_ctx_len is an upper bound on every ctx_len[s] (<= 0: max_pages_per_seq *
  * page_size); it fixes the chunking, so no host copy of the lengths is needed.
- * ctx_len[s] == 0 gives out = 0, lse = -inf.
+ * ctx_len[s] == 0 gives out = 0, lse = -inf.  A device length beyond what the launch was
+ * planned for (the chunks cover max_ctx_len rounded up to whole chunks, at most the block
+ * table's capacity) is clamped to that and sets EFIM_DEV_BAD_POSITION; nothing outside the
+ * workspace or the table is touched.
  */
 size_t efim_decode_workspace_bytes(const efim_cache_desc* cache, int32_t batch, int32_t max_ctx_len);
 /* Number of kernels the corresponding call enqueues for these arguments (the main
@@ -193,7 +235,9 @@ efim_status efim_decode_attn(const efim_cache_desc* cache, int32_t batch,
  * bit for bit, with one kernel less per step.  Differences: d_q is read only (the rotated q
  * is not written back); `rope` may be NULL or hold a NULL table (no rotation); rows with
  * ctx_len[s] == 0 append nothing.  A position >= rope->max_position sets
- * EFIM_DEV_BAD_POSITION and skips the row.  d_k_new / d_v_new: [batch][num_kv_heads][head_dim]
+ * EFIM_DEV_BAD_POSITION and skips the row (nothing appended, out = 0, lse = -inf); a length
+ * that had to be clamped (see efim_decode_attn) appends nothing either and attends over the
+ * clamped range.  d_k_new / d_v_new: [batch][num_kv_heads][head_dim]
  * bf16.  Workspace and every other argument as for efim_decode_attn.
  */
 efim_status efim_decode_step(const efim_cache_desc* cache, int32_t batch,
@@ -232,6 +276,16 @@ efim_status efim_decode_attn_static(const efim_cache_desc* cache, int32_t batch,
                                     const int32_t* d_block_table, int32_t max_pages_per_seq,
                                     const void* d_q, void* d_out, float* d_lse, float sm_scale,
                                     int32_t* d_status, void* stream);
+
+/*
+ * Self-test of the bounded device wait (the paper has no counterpart).  Every wait inside
+ * the kernels - on a bulk copy, on a tensor-core commit - gives up after a limit, sets
+ * EFIM_DEV_TIMEOUT in *d_status and lets the kernel end normally.  This call runs that code
+ * in isolation: one warp waits on a barrier that nothing will ever complete, with nothing in
+ * flight, for limit_ns nanoseconds (1 .. 100,000,000).  Afterwards *d_status has
+ * EFIM_DEV_TIMEOUT set and *d_waited_ns (optional, device) holds how long the warp waited.
+ */
+efim_status efim_selftest_bounded_wait(uint64_t limit_ns, int32_t* d_status, uint64_t* d_waited_ns, void* stream);
 
 /* ------------------------------------------------------------------------------------
  * Host-side front end (no GPU work): what turns a stream of infilling requests into the

@@ -9,4 +9,5 @@ from .binding import (  # noqa: F401
     efim_prefill_workspace_bytes, efim_decode_workspace_bytes, efim_rope_table_build,
     efim_strerror, efim_version, efim_decode_attn_static, efim_decode_static_scratch_bytes,
     efim_prefill_launch_count, efim_decode_launch_count, Frontend, efim_prefill_plan, efim_decode_step,
+    efim_append_prefill_step, efim_selftest_bounded_wait,
 )

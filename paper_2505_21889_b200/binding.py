@@ -40,6 +40,7 @@ EXPORTS = ("efim_last_cuda_error", "efim_strerror", "efim_version", "efim_rope_t
            "efim_decode_static_scratch_bytes", "efim_decode_attn_static",
            "efim_prefill_launch_count", "efim_decode_launch_count",
            "efim_prefill_plan_bytes", "efim_prefill_plan", "efim_append_prefill_attn_planned", "efim_decode_step",
+           "efim_append_prefill_step", "efim_selftest_bounded_wait",
            "efim_fragment_cuts", "efim_fim_split",
            "efim_frontend_create", "efim_frontend_destroy", "efim_frontend_transform", "efim_frontend_admit",
            "efim_frontend_finish", "efim_frontend_stats")
@@ -81,6 +82,12 @@ def load_library():
     lib.efim_append_prefill_attn_planned.argtypes = [POINTER(_CacheDesc), POINTER(_BatchDesc), c_void_p, c_size_t,
                                                      c_int32, c_void_p, c_void_p, c_void_p, c_float, c_void_p, c_size_t,
                                                      c_void_p, c_void_p]
+    lib.efim_append_prefill_step.restype = ctypes.c_int
+    lib.efim_append_prefill_step.argtypes = [POINTER(_CacheDesc), POINTER(_BatchDesc), POINTER(_RopeDesc), c_void_p,
+                                             c_void_p, c_void_p, c_void_p, c_void_p, c_float, c_void_p, c_size_t,
+                                             c_int32, c_void_p, c_size_t, c_void_p, c_void_p]
+    lib.efim_selftest_bounded_wait.restype = ctypes.c_int
+    lib.efim_selftest_bounded_wait.argtypes = [ctypes.c_uint64, c_void_p, c_void_p, c_void_p]
     lib.efim_decode_workspace_bytes.restype = c_size_t
     lib.efim_decode_workspace_bytes.argtypes = [POINTER(_CacheDesc), c_int32, c_int32]
     lib.efim_decode_attn.restype = ctypes.c_int
@@ -246,6 +253,26 @@ def efim_append_prefill_attn(cache: Cache, batch: Batch, q, out, lse=None, sm_sc
                                                   _stream_ptr(stream))
     if st != 0:
         raise EfimError(st, "efim_append_prefill_attn")
+
+
+def efim_append_prefill_step(cache: Cache, batch: Batch, rope, q, k_new, v_new, out, lse=None, sm_scale=0.0,
+                             workspace=None, status=None, stream=None, plan=None, lists_resident=False):
+    """kv_append of the new tokens' k/v and append-prefill attention with q rotated on load
+    (q is not modified)."""
+    nbytes = 0 if workspace is None else workspace.numel() * workspace.element_size()
+    st = load_library().efim_append_prefill_step(
+        ctypes.byref(cache.desc), ctypes.byref(batch.desc), ctypes.byref(rope.desc) if rope is not None else None,
+        _ptr(q), _ptr(k_new), _ptr(v_new), _ptr(out), _ptr(lse), float(sm_scale),
+        plan.ctypes.data if plan is not None else None, plan.nbytes if plan is not None else 0,
+        1 if lists_resident else 0, _ptr(workspace), nbytes, _ptr(status), _stream_ptr(stream))
+    if st != 0:
+        raise EfimError(st, "efim_append_prefill_step")
+
+
+def efim_selftest_bounded_wait(limit_ns: int, status, waited_ns=None, stream=None):
+    st = load_library().efim_selftest_bounded_wait(int(limit_ns), _ptr(status), _ptr(waited_ns), _stream_ptr(stream))
+    if st != 0:
+        raise EfimError(st, "efim_selftest_bounded_wait")
 
 
 def efim_decode_workspace_bytes(cache: Cache, batch: int, max_ctx_len: int) -> int:

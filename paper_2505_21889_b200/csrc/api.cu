@@ -1,6 +1,7 @@
 // Status strings and version of the EFIM C ABI.
+#include <atomic>
 #include <cuda_runtime.h>
-#include "efim.h"
+#include "common.cuh"
 
 static thread_local int g_last_cuda_error = 0;
 
@@ -23,4 +24,28 @@ extern "C" const char* efim_strerror(efim_status s) {
   return "unknown status";
 }
 
-extern "C" int efim_version(void) { return 100; }
+extern "C" int efim_version(void) { return 200; }
+
+namespace efim {
+// SM count of the current device (the planners size their grids by it), remembered per
+// device; 148 (a B200) when no device can be asked, so that sizing queries still answer.
+int sm_count() {
+  constexpr int kMaxDevices = 64;
+  static std::atomic<int> cached[kMaxDevices];
+  int dev = 0, n = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess) {
+    cudaGetLastError();
+    return 148;
+  }
+  if (dev >= 0 && dev < kMaxDevices) {
+    const int c = cached[dev].load(std::memory_order_relaxed);
+    if (c > 0) return c;
+  }
+  if (cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || n <= 0) {
+    cudaGetLastError();
+    return 148;
+  }
+  if (dev >= 0 && dev < kMaxDevices) cached[dev].store(n, std::memory_order_relaxed);
+  return n;
+}
+}  // namespace efim

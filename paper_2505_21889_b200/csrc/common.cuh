@@ -19,11 +19,15 @@ extern "C" void efim_note_cuda_error(int code);
 
 namespace efim {
 
+// SM count of the current device, cached per device (api.cu)
+int sm_count();
+
 // Validation shared by every entry point: shapes the kernels are built for.
 inline efim_status check_cache(const efim_cache_desc* c) {
   if (!c || !c->d_k_pool || !c->d_v_pool) return EFIM_ERR_INVALID_ARG;
   if (c->num_pages <= 0 || c->num_q_heads <= 0 || c->num_kv_heads <= 0) return EFIM_ERR_INVALID_ARG;
   if (c->num_q_heads % c->num_kv_heads != 0) return EFIM_ERR_INVALID_ARG;
+  if (c->num_kv_heads > 32767) return EFIM_ERR_UNSUPPORTED;
   if (c->page_size != 16) return EFIM_ERR_UNSUPPORTED;
   if (c->head_dim != 64 && c->head_dim != 128) return EFIM_ERR_UNSUPPORTED;
   if ((reinterpret_cast<uintptr_t>(c->d_k_pool) & 127) || (reinterpret_cast<uintptr_t>(c->d_v_pool) & 127))
@@ -78,6 +82,38 @@ __device__ __forceinline__ uint64_t fmul2(uint64_t a, uint64_t b) {
   uint64_t d;
   asm("mul.rn.f32x2 %0, %1, %2;" : "=l"(d) : "l"(a), "l"(b));
   return d;
+}
+
+// ---- rotary embedding, as every kernel of the library applies it: fp32 FMA from the bf16
+// inputs and the fp32 cos/sin table, one rounding to bf16.  (The same instruction sequence
+// everywhere, so a q or k rotated by one kernel equals the one rotated by another bit for bit.)
+// Rotate 8 (a, b) pairs held in two 16-byte vectors: a' = a c - b s, b' = b c + a s.
+__device__ __forceinline__ void rotate8(uint4& va, uint4& vb, const float* c, const float* s) {
+  uint32_t* a = reinterpret_cast<uint32_t*>(&va);
+  uint32_t* b = reinterpret_cast<uint32_t*>(&vb);
+#pragma unroll
+  for (int i = 0; i < 4; ++i) {
+    float a0 = bf16lo(a[i]), a1 = bf16hi(a[i]);
+    float b0 = bf16lo(b[i]), b1 = bf16hi(b[i]);
+    float ra0 = fmaf(a0, c[2 * i], -(b0 * s[2 * i]));
+    float ra1 = fmaf(a1, c[2 * i + 1], -(b1 * s[2 * i + 1]));
+    float rb0 = fmaf(b0, c[2 * i], a0 * s[2 * i]);
+    float rb1 = fmaf(b1, c[2 * i + 1], a1 * s[2 * i + 1]);
+    a[i] = pack_bf16x2(ra0, ra1);
+    b[i] = pack_bf16x2(rb0, rb1);
+  }
+}
+
+// Interleaved pairing: one 16-byte vector holds 4 pairs (2f, 2f+1).
+__device__ __forceinline__ void rotate4_interleaved(uint4& v, const float* c, const float* s) {
+  uint32_t* w = reinterpret_cast<uint32_t*>(&v);
+#pragma unroll
+  for (int i = 0; i < 4; ++i) {
+    float a = bf16lo(w[i]), b = bf16hi(w[i]);
+    float ra = fmaf(a, c[i], -(b * s[i]));
+    float rb = fmaf(b, c[i], a * s[i]);
+    w[i] = pack_bf16x2(ra, rb);
+  }
 }
 
 __device__ __forceinline__ uint4 ldg_stream(const void* p) {

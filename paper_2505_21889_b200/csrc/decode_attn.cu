@@ -8,6 +8,7 @@
 // copies (one per K page and V page).  Inside a warp D/8 lanes share one token
 // row (16 bytes each), so 32/(D/8) tokens are read per 128-bit shared-memory load.
 #include "decode_attn.cuh"
+#include "mbar.cuh"
 #include <algorithm>
 
 namespace efim {
@@ -46,18 +47,6 @@ __device__ __forceinline__ void transposed_reduce(float* x, int j) {
 // per SM it ran at 84 % of the measured copy bandwidth, with two and three at 99 %).
 constexpr int DEC_STAGES = 2;
 
-__device__ __forceinline__ uint32_t dec_smem_u32(const void* p) {
-  return static_cast<uint32_t>(__cvta_generic_to_shared(p));
-}
-__device__ __forceinline__ uint32_t dec_mbar_try(uint32_t bar, uint32_t parity) {
-  uint32_t ok;
-  asm volatile(
-      "{\n.reg .pred p;\nmbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\nselp.u32 %0, 1, 0, p;\n}\n"
-      : "=r"(ok)
-      : "r"(bar), "r"(parity)
-      : "memory");
-  return ok;
-}
 __device__ __forceinline__ void dec_bulk_load(uint32_t dst, const void* src, uint32_t bytes, uint32_t bar) {
   asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];" ::"r"(dst),
                "l"(src), "r"(bytes), "r"(bar)
@@ -130,8 +119,13 @@ __global__ void __launch_bounds__(128, 3) decode_splitkv_kernel(const DecodePara
   const int my_pg = first_pg + 4 * (threadIdx.x & 31);
   const int pid_early = my_pg < p.max_pages_per_seq ? __ldg(bt + my_pg) : -1;
   int len = __ldg(p.row_len + r);
-  if (len > p.max_pages_per_seq * 16) {           // longer than the block table can address: clamp and report
-    len = p.max_pages_per_seq * 16;
+  // longer than the launch was planned for (max_ctx_len) or than the block table can address:
+  // clamp and report.  A fused step then has no valid position for its new token and runs as a
+  // plain decode over the clamped range.
+  bool append = FUSED;
+  if (len > p.key_cap) {
+    len = p.key_cap;
+    append = false;
     if (threadIdx.x == 0 && p.status) atomicOr(p.status, EFIM_DEV_BAD_POSITION);
   }
   const int begin = c * p.chunk_tokens;
@@ -139,18 +133,31 @@ __global__ void __launch_bounds__(128, 3) decode_splitkv_kernel(const DecodePara
   const int tid = threadIdx.x;
   // fused step: the new token sits at position len - 1; its rotation needs a table row
   const float* cs_row = nullptr;
-  if (FUSED && len > 0 && p.cos_sin) {
+  bool skip_row = false;
+  if (FUSED && append && len > 0 && p.cos_sin) {
     if (len - 1 >= p.max_position) {
+      // no table row for the new token's position: report it and skip the row (nothing is
+      // appended; the output is zero, lse -inf)
       if (tid == 0 && p.status) atomicOr(p.status, EFIM_DEV_BAD_POSITION);
-      return;
+      skip_row = true;
+    } else {
+      cs_row = p.cos_sin + (size_t)(len - 1) * D;
     }
-    cs_row = p.cos_sin + (size_t)(len - 1) * D;
   }
-  if (begin >= len) {
-    // nothing visible in this chunk; a row without any key still gets a defined result
-    if (len <= 0 && c == 0 && p.n_chunks == 1) {
-      for (int i = tid; i < ng * D; i += 128) p.out[((size_t)r * p.Hq + head0) * D + i] = 0;
-      if (p.lse && tid < ng) p.lse[(size_t)r * p.Hq + head0 + tid] = -INFINITY;
+  if (begin >= len || skip_row) {
+    // nothing to attend in this chunk.  A row without any key (or a skipped one) still gets a
+    // defined result: directly, or as an empty partial for every chunk the merge will read.
+    if (p.n_chunks == 1) {
+      if (len <= 0 || skip_row) {
+        for (int i = tid; i < ng * D; i += 128) p.out[((size_t)r * p.Hq + head0) * D + i] = 0;
+        if (p.lse && tid < ng) p.lse[(size_t)r * p.Hq + head0 + tid] = -INFINITY;
+      }
+    } else if (skip_row && begin < len) {
+      for (int i = tid; i < ng * D; i += 128) {
+        const size_t row_head = (size_t)r * p.Hq + head0 + i / D;
+        p.part_o[(row_head * p.n_chunks + c) * D + i % D] = 0.f;
+        if (i % D == 0) p.part_lse[row_head * p.n_chunks + c] = -INFINITY;
+      }
     }
     return;
   }
@@ -164,8 +171,8 @@ __global__ void __launch_bounds__(128, 3) decode_splitkv_kernel(const DecodePara
   uint8_t* ring = dec_ring + warp * (DEC_STAGES * 2 * PAGE_BYTES);
   if (lane == 0) {
     for (int sg = 0; sg < DEC_STAGES; ++sg)
-      asm volatile("mbarrier.init.shared::cta.b64 [%0], 1;" ::"r"(dec_smem_u32(&s_bar[warp][sg])) : "memory");
-    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+      mbar_init(smem_u32(&s_bar[warp][sg]), 1);
+    mbar_fence_init();
   }
   __syncwarp();
   // page ids of the next 32 pages of this warp, one per lane (refilled every 32 pages)
@@ -174,9 +181,9 @@ __global__ void __launch_bounds__(128, 3) decode_splitkv_kernel(const DecodePara
     const int pid = __shfl_sync(0xffffffffu, pid_cache, i & 31);
     const bool ok = pid >= 0 && pid < p.num_pages;
     if (lane == 0) {
-      const uint32_t bar = dec_smem_u32(&s_bar[warp][i % DEC_STAGES]);
+      const uint32_t bar = smem_u32(&s_bar[warp][i % DEC_STAGES]);
       if (ok) {
-        const uint32_t dst = dec_smem_u32(ring + (i % DEC_STAGES) * 2 * PAGE_BYTES);
+        const uint32_t dst = smem_u32(ring + (i % DEC_STAGES) * 2 * PAGE_BYTES);
         const size_t off = ((size_t)pid * p.Hkv + kvh) * 16 * D;
         asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(2 * PAGE_BYTES) : "memory");
         dec_bulk_load(dst, p.k_pool + off, PAGE_BYTES, bar);
@@ -223,34 +230,22 @@ __global__ void __launch_bounds__(128, 3) decode_splitkv_kernel(const DecodePara
 
   const int odd = j & 1;
   const int st_mine = j >> 1;                   // step whose scores this lane ends up with
-  bool gave_up = false;
+  int gave_up_at = -1;                          // page index at which a stage wait expired
 
   for (int i = 0; i < n_pages; ++i) {
     const int pg = first_pg + 4 * i;
     const int sg = i % DEC_STAGES;
     const bool page_ok = (ok_bits >> sg) & 1u;
-    // ---- wait for the stage (bounded: ~2 s, then flag and stop)
+    // ---- wait for the stage (bounded; on expiry flag and stop walking)
     {
-      const uint32_t bar = dec_smem_u32(&s_bar[warp][sg]);
-      const uint32_t parity = (i / DEC_STAGES) & 1;
-      if (!dec_mbar_try(bar, parity)) {
-        unsigned long long t0, t1;
-        asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t0));
-        uint32_t spins = 0;
-        while (!dec_mbar_try(bar, parity)) {
-          if ((++spins & 1023u) == 0) {
-            asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t1));
-            if (t1 - t0 > 2000000000ull) { gave_up = true; break; }
-          }
-        }
-      }
-      gave_up = __any_sync(0xffffffffu, gave_up);
-      if (gave_up) {
-        if (lane == 0 && p.status) atomicOr(p.status, EFIM_DEV_TIMEOUT);
+      const bool ok = mbar_wait_bounded(smem_u32(&s_bar[warp][sg]), (i / DEC_STAGES) & 1, p.wait_ns, nullptr,
+                                        lane == 0 ? p.status : nullptr);
+      if (__any_sync(0xffffffffu, !ok)) {
+        gave_up_at = i;
         break;
       }
     }
-    if (FUSED && page_ok && pg == ((len - 1) >> 4)) {
+    if (FUSED && append && page_ok && pg == ((len - 1) >> 4)) {
       // The page of the new token: whatever the copy brought for its slot is replaced, in
       // shared memory, by the token's rotated k and its v; the CTA of the kv head's first
       // group tile also puts them into the pools.  (Other CTAs that read this page patch
@@ -368,6 +363,12 @@ __global__ void __launch_bounds__(128, 3) decode_splitkv_kernel(const DecodePara
     }
   }
 
+  if (gave_up_at >= 0) {
+    // copies issued for the stages still in flight must land before the CTA's shared memory
+    // can be handed to another CTA
+    for (int k = gave_up_at; k < min(gave_up_at + DEC_STAGES, n_pages); ++k)
+      mbar_drain(smem_u32(&s_bar[warp][k % DEC_STAGES]), (k / DEC_STAGES) & 1);
+  }
   float o[GT][8];
 #pragma unroll
   for (int g = 0; g < GT; ++g)
@@ -430,7 +431,7 @@ __global__ void __launch_bounds__(128) decode_merge_kernel(const DecodeParams p)
   const size_t row_head = (size_t)blockIdx.x * 4 + (threadIdx.x >> 5);
   if (row_head >= (size_t)p.R * p.Hq) return;
   const int r = (int)(row_head / p.Hq);
-  const int len = min(__ldg(p.row_len + r), p.max_pages_per_seq * 16);
+  const int len = min(__ldg(p.row_len + r), p.key_cap);
   uint16_t* out = p.out + row_head * D + lane * EPL;
   if (len <= 0) {
 #pragma unroll
@@ -438,7 +439,7 @@ __global__ void __launch_bounds__(128) decode_merge_kernel(const DecodeParams p)
     if (p.lse && lane == 0) p.lse[row_head] = -INFINITY;
     return;
   }
-  const int nc = (len + p.chunk_tokens - 1) / p.chunk_tokens;
+  const int nc = min((len + p.chunk_tokens - 1) / p.chunk_tokens, p.n_chunks);
   const float* pl = p.part_lse + row_head * p.n_chunks;
   const float* po = p.part_o + row_head * p.n_chunks * D + lane * EPL;
   // the lanes fetch the chunks' lse values side by side; the partial rows are then loaded four
@@ -449,6 +450,12 @@ __global__ void __launch_bounds__(128) decode_merge_kernel(const DecodeParams p)
     if (c0 + lane < nc) M = fmaxf(M, __ldg(pl + c0 + lane));
 #pragma unroll
   for (int d = 16; d > 0; d >>= 1) M = fmaxf(M, __shfl_xor_sync(0xffffffffu, M, d));
+  if (M == -INFINITY) {                            // every chunk came back empty (a skipped row)
+#pragma unroll
+    for (int e = 0; e < EPL; ++e) out[e] = 0;
+    if (p.lse && lane == 0) p.lse[row_head] = -INFINITY;
+    return;
+  }
   float L = 0.f, acc[EPL];
 #pragma unroll
   for (int e = 0; e < EPL; ++e) acc[e] = 0.f;
@@ -494,14 +501,15 @@ DecodePlan plan_decode(int rows, int Hq, int Hkv, int D, int max_len) {
   // a few microseconds before its pages stream, and shorter chunks were measured slower
   // (16 rows x 8 kv heads x 2.5k keys: 48.9 us per step with 256-key chunks, 43 with 768).
   // Only when that leaves fewer than two CTAs per SM do the chunks shrink, down to 256.
+  const long long n_sm = sm_count();
   const long long ctas_per_chunkless = (long long)rows * Hkv * pl.gsplit;
-  long long want_chunks = (148LL * 32 + ctas_per_chunkless - 1) / ctas_per_chunkless;
+  long long want_chunks = (n_sm * 32 + ctas_per_chunkless - 1) / ctas_per_chunkless;
   if (want_chunks < 1) want_chunks = 1;
   long long chunk = (max_len + want_chunks - 1) / want_chunks;
   if (chunk < 768) chunk = 768;
   if (chunk > 2048) chunk = 2048;
-  if (ctas_per_chunkless * ((max_len + chunk - 1) / chunk) < 148LL * 2) {
-    const long long need_chunks = (148LL * 2 + ctas_per_chunkless - 1) / ctas_per_chunkless;
+  if (ctas_per_chunkless * ((max_len + chunk - 1) / chunk) < n_sm * 2) {
+    const long long need_chunks = (n_sm * 2 + ctas_per_chunkless - 1) / ctas_per_chunkless;
     chunk = std::max<long long>(256, (max_len + need_chunks - 1) / need_chunks);
     if (chunk > 2048) chunk = 2048;
   }
@@ -568,12 +576,11 @@ extern "C" int32_t efim_decode_launch_count(const efim_cache_desc* cache, int32_
   return pl.n_chunks > 1 ? 2 : 1;
 }
 
-// efim_decode_attn, and efim_decode_step when d_k_new / d_v_new are given
-static efim_status decode_entry(const efim_cache_desc* cache, int32_t batch, const int32_t* d_ctx_len,
-                                int32_t max_ctx_len, const int32_t* d_block_table, int32_t max_pages_per_seq,
-                                const efim_rope_desc* rope, const void* d_k_new, const void* d_v_new, bool fused,
-                                const void* d_q, void* d_out, float* d_lse, float sm_scale, void* d_workspace,
-                                size_t workspace_bytes, int32_t* d_status, void* stream) {
+efim_status efim::decode_run(const efim_cache_desc* cache, int32_t batch, const int32_t* d_ctx_len,
+                             int32_t max_ctx_len, const int32_t* d_block_table, int32_t max_pages_per_seq,
+                             const efim_rope_desc* rope, const void* d_k_new, const void* d_v_new, bool fused,
+                             const void* d_q, void* d_out, float* d_lse, float sm_scale, void* d_workspace,
+                             size_t workspace_bytes, int32_t* d_status, void* stream, WorkspaceSource ws_source) {
   efim_status st = efim::check_cache(cache);
   if (st != EFIM_OK) return st;
   if (batch < 0 || max_pages_per_seq <= 0) return EFIM_ERR_INVALID_ARG;
@@ -587,6 +594,10 @@ static efim_status decode_entry(const efim_cache_desc* cache, int32_t batch, con
                                                 max_ctx_len);
   const size_t need = pl.part_o_bytes + pl.part_lse_bytes;
   if (need > 0) {
+    if (ws_source) {
+      st = ws_source(&d_workspace, &workspace_bytes);
+      if (st != EFIM_OK) return st;
+    }
     if (!d_workspace || workspace_bytes < need) return EFIM_ERR_WORKSPACE;
     if (reinterpret_cast<uintptr_t>(d_workspace) & 255) return EFIM_ERR_INVALID_ARG;
   }
@@ -609,6 +620,8 @@ static efim_status decode_entry(const efim_cache_desc* cache, int32_t batch, con
   p.num_pages = cache->num_pages;
   p.chunk_tokens = pl.chunk_tokens;
   p.n_chunks = pl.n_chunks;
+  p.key_cap = (int)std::min<long long>((long long)pl.n_chunks * pl.chunk_tokens, cap);
+  p.wait_ns = efim::WAIT_LIMIT_NS;
   const float scale = sm_scale > 0.f ? sm_scale : 1.0f / sqrtf((float)cache->head_dim);
   p.scale_log2 = scale * 1.4426950408889634f;
   if (fused) {
@@ -634,7 +647,7 @@ extern "C" efim_status efim_decode_attn(const efim_cache_desc* cache, int32_t ba
                                         int32_t max_pages_per_seq, const void* d_q, void* d_out, float* d_lse,
                                         float sm_scale, void* d_workspace, size_t workspace_bytes,
                                         int32_t* d_status, void* stream) {
-  return decode_entry(cache, batch, d_ctx_len, max_ctx_len, d_block_table, max_pages_per_seq, nullptr, nullptr,
+  return efim::decode_run(cache, batch, d_ctx_len, max_ctx_len, d_block_table, max_pages_per_seq, nullptr, nullptr,
                       nullptr, false, d_q, d_out, d_lse, sm_scale, d_workspace, workspace_bytes, d_status, stream);
 }
 
@@ -644,6 +657,6 @@ extern "C" efim_status efim_decode_step(const efim_cache_desc* cache, int32_t ba
                                         const void* d_k_new, const void* d_v_new, void* d_out, float* d_lse,
                                         float sm_scale, void* d_workspace, size_t workspace_bytes,
                                         int32_t* d_status, void* stream) {
-  return decode_entry(cache, batch, d_ctx_len, max_ctx_len, d_block_table, max_pages_per_seq, rope, d_k_new,
+  return efim::decode_run(cache, batch, d_ctx_len, max_ctx_len, d_block_table, max_pages_per_seq, rope, d_k_new,
                       d_v_new, true, d_q, d_out, d_lse, sm_scale, d_workspace, workspace_bytes, d_status, stream);
 }

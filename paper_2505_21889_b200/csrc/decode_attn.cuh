@@ -18,6 +18,9 @@ struct DecodeParams {
   float* part_lse;            // [R][Hq][n_chunks]      base-2 log
   int32_t* status;
   int R, Hq, Hkv, max_pages_per_seq, num_pages, chunk_tokens, n_chunks;
+  int key_cap;                // keys the launch can cover: min(n_chunks * chunk_tokens, table capacity);
+                              // a longer device length is clamped to it and reported
+  unsigned long long wait_ns; // limit of every device-side wait
   float scale_log2;           // sm_scale * log2(e)
   // fused decode step: the row's last key (position row_len[r] - 1) is this step's new token.
   // Its k/v are rotated, put into the page slot and used from shared memory in the same
@@ -40,5 +43,16 @@ struct DecodePlan {
 
 DecodePlan plan_decode(int rows, int Hq, int Hkv, int D, int max_len);
 efim_status launch_decode(const DecodeParams& p, const DecodePlan& pl, int D, cudaStream_t s);
+
+// Validation, planning and launch behind efim_decode_attn, efim_decode_step (fused = true:
+// rope / d_k_new / d_v_new are used) and efim_decode_attn_static.  The latter passes a
+// `ws_source`: asked, once the arguments have passed validation and only if the plan needs
+// partials, for the workspace to use (the library's fixed array) in place of the caller's.
+typedef efim_status (*WorkspaceSource)(void** d_workspace, size_t* workspace_bytes);
+efim_status decode_run(const efim_cache_desc* cache, int32_t batch, const int32_t* d_ctx_len, int32_t max_ctx_len,
+                       const int32_t* d_block_table, int32_t max_pages_per_seq, const efim_rope_desc* rope,
+                       const void* d_k_new, const void* d_v_new, bool fused, const void* d_q, void* d_out,
+                       float* d_lse, float sm_scale, void* d_workspace, size_t workspace_bytes, int32_t* d_status,
+                       void* stream, WorkspaceSource ws_source = nullptr);
 
 }  // namespace efim

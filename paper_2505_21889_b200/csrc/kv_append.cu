@@ -22,35 +22,6 @@ struct KvAppendParams {
   int num_pages, Hq, Hkv, max_position, interleaved;
 };
 
-// Rotate 8 (a, b) pairs held in two 16-byte vectors: a' = a c - b s, b' = b c + a s.
-__device__ __forceinline__ void rotate8(uint4& va, uint4& vb, const float* c, const float* s) {
-  uint32_t* a = reinterpret_cast<uint32_t*>(&va);
-  uint32_t* b = reinterpret_cast<uint32_t*>(&vb);
-#pragma unroll
-  for (int i = 0; i < 4; ++i) {
-    float a0 = bf16lo(a[i]), a1 = bf16hi(a[i]);
-    float b0 = bf16lo(b[i]), b1 = bf16hi(b[i]);
-    float ra0 = fmaf(a0, c[2 * i], -(b0 * s[2 * i]));
-    float ra1 = fmaf(a1, c[2 * i + 1], -(b1 * s[2 * i + 1]));
-    float rb0 = fmaf(b0, c[2 * i], a0 * s[2 * i]);
-    float rb1 = fmaf(b1, c[2 * i + 1], a1 * s[2 * i + 1]);
-    a[i] = pack_bf16x2(ra0, ra1);
-    b[i] = pack_bf16x2(rb0, rb1);
-  }
-}
-
-// Interleaved pairing: one 16-byte vector holds 4 pairs (2f, 2f+1).
-__device__ __forceinline__ void rotate4_interleaved(uint4& v, const float* c, const float* s) {
-  uint32_t* w = reinterpret_cast<uint32_t*>(&v);
-#pragma unroll
-  for (int i = 0; i < 4; ++i) {
-    float a = bf16lo(w[i]), b = bf16hi(w[i]);
-    float ra = fmaf(a, c[i], -(b * s[i]));
-    float rb = fmaf(b, c[i], a * s[i]);
-    w[i] = pack_bf16x2(ra, rb);
-  }
-}
-
 // WPT warps per new token, 256 threads per CTA.  A lane keeps one position along the head
 // dimension (vector j, and for the rotate-half pairing its partner j + D/16), so its
 // cos/sin values are loaded once, and walks the heads - q heads (rotated in place), then

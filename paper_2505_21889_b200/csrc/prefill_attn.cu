@@ -5,6 +5,7 @@
 #include <cstring>
 #include <vector>
 #include "prefill_tc.cuh"
+#include "mbar.cuh"
 
 extern "C" size_t efim_prefill_workspace_bytes(const efim_cache_desc* cache, const efim_batch_desc* batch) {
   if (efim::check_cache(cache) != EFIM_OK || efim::check_batch(cache, batch, true) != EFIM_OK) return 0;
@@ -93,11 +94,12 @@ extern "C" efim_status efim_prefill_plan(const efim_cache_desc* cache, const efi
   return EFIM_OK;
 }
 
-extern "C" efim_status efim_append_prefill_attn_planned(const efim_cache_desc* cache, const efim_batch_desc* batch,
-                                                        const void* h_plan, size_t plan_bytes,
-                                                        int32_t lists_resident, const void* d_q, void* d_out,
-                                                        float* d_lse, float sm_scale, void* d_workspace,
-                                                        size_t workspace_bytes, int32_t* d_status, void* stream) {
+namespace {
+// Runs a plan.  `rope` with a table: the query rows are rotated as the kernel loads them.
+efim_status run_planned(const efim_cache_desc* cache, const efim_batch_desc* batch, const efim_rope_desc* rope,
+                        const void* h_plan, size_t plan_bytes, int32_t lists_resident, const void* d_q, void* d_out,
+                        float* d_lse, float sm_scale, void* d_workspace, size_t workspace_bytes, int32_t* d_status,
+                        void* stream) {
   using namespace efim;
   efim_status st = check_cache(cache);
   if (st != EFIM_OK) return st;
@@ -153,14 +155,20 @@ extern "C" efim_status efim_append_prefill_attn_planned(const efim_cache_desc* c
   p.s_max = pl.s_max;
   const float scale = sm_scale > 0.f ? sm_scale : 1.0f / sqrtf((float)cache->head_dim);
   p.scale_log2 = scale * 1.4426950408889634f;
+  p.wait_ns = WAIT_LIMIT_NS;
+  if (rope && rope->d_cos_sin) {
+    if (rope->max_position <= 0 || (reinterpret_cast<uintptr_t>(rope->d_cos_sin) & 15)) return EFIM_ERR_INVALID_ARG;
+    p.cos_sin = rope->d_cos_sin;
+    p.max_position = rope->max_position;
+    p.interleaved = rope->interleaved;
+  }
   return pf::launch(cache, p, pl, s);
 }
 
-// Plan and run in one call.
-extern "C" efim_status efim_append_prefill_attn(const efim_cache_desc* cache, const efim_batch_desc* batch,
-                                                const void* d_q, void* d_out, float* d_lse, float sm_scale,
-                                                void* d_workspace, size_t workspace_bytes, int32_t* d_status,
-                                                void* stream) {
+// Plans into a temporary blob, then runs it.
+efim_status plan_and_run(const efim_cache_desc* cache, const efim_batch_desc* batch, const efim_rope_desc* rope,
+                         const void* d_q, void* d_out, float* d_lse, float sm_scale, void* d_workspace,
+                         size_t workspace_bytes, int32_t* d_status, void* stream) {
   using namespace efim;
   efim_status st = check_cache(cache);
   if (st != EFIM_OK) return st;
@@ -170,6 +178,44 @@ extern "C" efim_status efim_append_prefill_attn(const efim_cache_desc* cache, co
   const pf::Plan sized = pf::make_plan(cache, batch, nullptr, nullptr);
   std::vector<unsigned char> blob(PLAN_HEAD_BYTES + sized.items_bytes + sized.split_bytes);
   fill_plan(cache, batch, &sized, blob.data());
-  return efim_append_prefill_attn_planned(cache, batch, blob.data(), blob.size(), 0, d_q, d_out, d_lse, sm_scale,
-                                          d_workspace, workspace_bytes, d_status, stream);
+  return run_planned(cache, batch, rope, blob.data(), blob.size(), 0, d_q, d_out, d_lse, sm_scale, d_workspace,
+                     workspace_bytes, d_status, stream);
+}
+}  // namespace
+
+extern "C" efim_status efim_append_prefill_attn_planned(const efim_cache_desc* cache, const efim_batch_desc* batch,
+                                                        const void* h_plan, size_t plan_bytes,
+                                                        int32_t lists_resident, const void* d_q, void* d_out,
+                                                        float* d_lse, float sm_scale, void* d_workspace,
+                                                        size_t workspace_bytes, int32_t* d_status, void* stream) {
+  return run_planned(cache, batch, nullptr, h_plan, plan_bytes, lists_resident, d_q, d_out, d_lse, sm_scale,
+                     d_workspace, workspace_bytes, d_status, stream);
+}
+
+// Plan and run in one call.
+extern "C" efim_status efim_append_prefill_attn(const efim_cache_desc* cache, const efim_batch_desc* batch,
+                                                const void* d_q, void* d_out, float* d_lse, float sm_scale,
+                                                void* d_workspace, size_t workspace_bytes, int32_t* d_status,
+                                                void* stream) {
+  return plan_and_run(cache, batch, nullptr, d_q, d_out, d_lse, sm_scale, d_workspace, workspace_bytes, d_status,
+                      stream);
+}
+
+// Steps 1 and 2 of a turn: the new tokens' k/v go into the pages (k rotated), then the new
+// queries, rotated as they are loaded, attend over everything before them.
+extern "C" efim_status efim_append_prefill_step(const efim_cache_desc* cache, const efim_batch_desc* batch,
+                                                const efim_rope_desc* rope, const void* d_q, const void* d_k_new,
+                                                const void* d_v_new, void* d_out, float* d_lse, float sm_scale,
+                                                const void* h_plan, size_t plan_bytes, int32_t lists_resident,
+                                                void* d_workspace, size_t workspace_bytes, int32_t* d_status,
+                                                void* stream) {
+  if ((d_k_new == nullptr) != (d_v_new == nullptr)) return EFIM_ERR_INVALID_ARG;
+  if (d_k_new) {
+    const efim_status st = efim_kv_append(cache, batch, rope, nullptr, d_k_new, d_v_new, d_status, stream);
+    if (st != EFIM_OK) return st;
+  }
+  if (h_plan)
+    return run_planned(cache, batch, rope, h_plan, plan_bytes, lists_resident, d_q, d_out, d_lse, sm_scale,
+                       d_workspace, workspace_bytes, d_status, stream);
+  return plan_and_run(cache, batch, rope, d_q, d_out, d_lse, sm_scale, d_workspace, workspace_bytes, d_status, stream);
 }

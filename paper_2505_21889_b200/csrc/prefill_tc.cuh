@@ -18,12 +18,19 @@ constexpr int REGS_SOFTMAX = 216;
 constexpr int REGS_SERVICE = 64;
 
 // One CTA's work: packed rows [row0, row0 + 256) of (seq, kv head) against KV tiles
-// [tile_begin, tile_end).  Packed row R = token * G + head-in-group.
+// [tile_begin, tile_end).  Packed row R = token * G + head-in-group.  The sequence's
+// lengths and first query row ride along (the planner has them from the host mirrors),
+// so that a CTA's first dependent chain is "item -> block table / query rows" instead of
+// "item -> lengths -> block table / query rows".
 struct WorkItem {
-  int32_t seq, kvh, row0, tile_begin, tile_end;
-  int32_t chunk;               // >= 0: write a partial for this KV chunk; -1: final output
-  int32_t pad0, pad1;
+  int32_t seq;
+  int16_t kvh;
+  int16_t chunk;               // >= 0: write a partial for this KV chunk; -1: final output
+  int32_t row0, tile_begin, tile_end;
+  int32_t cached, new_len;     // cached_len[seq], new_len[seq]
+  int32_t tok0;                // q_indptr[seq]
 };
+static_assert(sizeof(WorkItem) == 32, "work items are read as two 16-byte vectors");
 
 struct Params {
   const uint16_t* q;           // [T][Hq][D]
@@ -41,6 +48,10 @@ struct Params {
   int batch, total_new_tokens;
   int Hq, Hkv, G, max_pages_per_seq, num_pages, s_max;
   float scale_log2;
+  unsigned long long wait_ns;  // limit of every device-side wait
+  // rotation of the query rows as they are loaded (null: q is already rotated)
+  const float* cos_sin;        // [max_position][D]
+  int max_position, interleaved;
 };
 
 struct Plan {

@@ -12,7 +12,10 @@ from oracle import efim_oracle as orc
 # spec tolerances for bf16 attention outputs with fp32 accumulation
 MAX_ABS_TOL = 2e-2
 MEAN_ABS_TOL = 2e-3
-LSE_TOL = 2e-3
+# lse: 1e-3 absolute.  The largest error seen over all cases, full sizes included, is 4.2e-4
+# (rows with thousands of keys; the scores leave the tensor core with ~1e-4 of absolute error
+# at |score| ~ 10), the decode kernel's fp32 FMA chains stay below 3e-5.
+LSE_TOL = 1e-3
 
 
 def bits_to_torch(bits: np.ndarray, device="cuda"):
@@ -47,8 +50,17 @@ def assert_attn_close(got_bf16_bits, want_f64, what):
     got = bf16_bits_to_f32(got_bf16_bits).astype(np.float64)
     err = np.abs(got - want_f64)
     assert np.isfinite(got).all(), f"{what}: non-finite output"
+    print(f"out max abs err {err.max(initial=0):.3e} mean {err.mean() if err.size else 0.0:.3e}  [{what}]")
     assert err.max(initial=0) <= MAX_ABS_TOL, f"{what}: max abs err {err.max():.4g}"
     assert err.mean() <= MEAN_ABS_TOL, f"{what}: mean abs err {err.mean():.4g}"
+
+
+def assert_lse_close(got, want, what):
+    """|lse error| against the fp64 oracle; the figure is printed so a run with -rP shows the
+    margin every case leaves."""
+    err = float(np.abs(np.asarray(got, np.float64) - want).max(initial=0))
+    print(f"lse max abs err {err:.3e}  [{what}]")
+    assert err <= LSE_TOL, f"{what}: lse max abs err {err:.4g}"
 
 
 class DeviceWorkload:

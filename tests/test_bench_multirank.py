@@ -51,3 +51,32 @@ def test_workload_counts_match_definitions():
     assert c["prefill_flops"] == 4 * 128 * 32 * pairs
     assert c["prefill_kv_bytes"] == 4 * 128 * 8 * 8 * (8192 + 128)
     assert c["kv_append_bytes_per_token"] == 4 * 128 * (32 + 16)
+
+
+def test_plain_run_with_gpus_2_starts_two_ranks():
+    """`python bench.py --gpus 2` without a launcher starts the two ranks itself; with
+    --selfcheck-ranks they run the rank plumbing on CPU (gloo) with a stand-in measurement."""
+    import json
+    import subprocess
+    env = {k: v for k, v in os.environ.items() if k not in ("WORLD_SIZE", "RANK", "LOCAL_RANK")}
+    res = subprocess.run([sys.executable, os.path.join(ROOT, "bench.py"), "--gpus", "2", "--selfcheck-ranks"],
+                         capture_output=True, text=True, timeout=300, env=env)
+    assert res.returncode == 0, res.stderr[-2000:]
+    lines = [ln for ln in res.stdout.splitlines() if ln.startswith("{")]
+    assert len(lines) == 1                       # rank 0 alone prints
+    out = json.loads(lines[0])
+    assert out["n_gpus"] == 2 and out["ms"] == 15.0 and out["tokens"] == 3000.0
+
+
+def test_reference_arm_prints_the_contract_line_on_the_native_config():
+    import json
+    import subprocess
+    res = subprocess.run([sys.executable, os.path.join(ROOT, "bench.py"), "--impl", "reference", "--workload", "cfg1",
+                          "--steps", "2", "--warmup", "1"], capture_output=True, text=True, timeout=600)
+    assert res.returncode == 0, res.stderr[-2000:]
+    out = json.loads([ln for ln in res.stdout.splitlines() if ln.startswith("{")][-1])
+    import bench
+    from efim_synth import make_workload
+    assert out["impl"] == "reference" and out["config"] == bench.config_of(make_workload("cfg1"), 1)
+    assert out["e2e"]["value"] == out["value"] and out["cpu_baseline"]["kind"] == "oracle"
+    assert out["steps"] == 2 and out["warmup"] == 1 and out["gpu_launches"] == 0

@@ -1,6 +1,7 @@
 """Parity at the full sizes of the five configs, in the launch configuration bench.py
-times.  The GPU processes the whole batch; the oracle recomputes sampled sequences
-(and, for the long FIM-miss rows, sampled token windows) from the same seeded bytes."""
+times.  The GPU processes the whole batch; the oracle recomputes every row of cfg2, cfg3
+and cfg4a, every row of one cfg4b sequence plus token windows of others, and 16 sequences
+of cfg5 at decode steps 0, 31 and 63, from the same seeded bytes."""
 import numpy as np
 import pytest
 import torch
@@ -26,48 +27,45 @@ def _run_turn(w, seqs, windows=None):
         H.assert_rope_close(dw.pages_from_device("k", pg), ref["k_pool"][ref["bt"][r, :len(pg)]], f"{w.name} K pages")
     H.assert_rope_close(H.torch_to_bits(dw.q)[ref["rows"]], ref["q_rot"], f"{w.name} q")
     H.assert_attn_close(H.torch_to_bits(dw.out)[ref["attn_rows"]], ref["o"], f"{w.name} full size")
-    assert np.abs(dw.lse.cpu().numpy()[ref["attn_rows"]] - ref["lse"]).max() <= H.LSE_TOL
+    H.assert_lse_close(dw.lse.cpu().numpy()[ref["attn_rows"]], ref["lse"], f"{w.name} full size")
     # every output of the batch is finite (also the rows the oracle did not recompute)
     assert torch.isfinite(dw.out.float()).all()
     return dw, ref
 
 
-def test_cfg2_full_sampled_sequences():
-    w = make_workload("cfg2")
-    order = np.argsort(w.cached_len + w.new_len)
-    _run_turn(w, sorted([int(order[0]), int(order[-1]), int(order[7])]))
+@pytest.mark.parametrize("name", ["cfg2", "cfg3", "cfg4a"])
+def test_full_size_all_rows(name):
+    """Every row of the batch against the oracle (cfg3: its 32 prefill rows and its 32
+    one-token decode rows, all through the prefill call)."""
+    _run_turn(make_workload(name), None)
 
 
-def test_cfg3_full_sampled_rows():
-    w = make_workload("cfg3")
-    pre = np.where(~w.decode_rows)[0]
-    dec = np.where(w.decode_rows)[0]
-    L = w.cached_len + w.new_len
-    picks = [int(pre[np.argmin(L[pre])]), int(pre[np.argmax(w.new_len[pre])]), int(dec[np.argmax(L[dec])]),
-             int(dec[0])]
-    _run_turn(w, sorted(set(picks)))
-
-
-def test_cfg4a_full_one_sequence():
-    _run_turn(make_workload("cfg4a"), [3])
-
-
-@pytest.mark.parametrize("name", ["cfg4b", "cfg4b_3072"])
-def test_cfg4b_full_token_windows(name):
-    w = make_workload(name)
-    n = int(w.new_len[5])
-    # three windows of the recomputed suffix: start, middle (across a tile edge), end
+def test_cfg4b_full_one_sequence_all_rows_and_windows_of_others():
+    """The FIM-miss recompute: all 3,200 rows of one sequence, and of two other sequences the
+    first, a middle (across a row-tile edge) and the last window of 48 tokens."""
+    w = make_workload("cfg4b")
+    _run_turn(w, [5])
+    n = int(w.new_len[0])
     for first in (0, n // 2 - 24, n - 48):
-        _run_turn(w, [5], windows=[(first, 48)])
+        _run_turn(w, [0, 7], windows=[(first, 48), (first, 48)])
 
 
-def test_cfg5_full_decode_steps_sampled():
+def test_cfg4b_3072_full_token_windows():
+    w = make_workload("cfg4b_3072")
+    n = int(w.new_len[2])
+    for first in (0, n // 2 - 24, n - 48):
+        _run_turn(w, [2], windows=[(first, 48)])
+
+
+def test_cfg5_full_decode_steps_16_sequences():
     import tests.gpu_harness as H
     w = make_workload("cfg5")
     dw = H.DeviceWorkload(w)
     ctx_all = w.cached_len.astype(np.int32).copy()
     order = np.argsort(ctx_all)
-    seqs = sorted([int(order[0]), int(order[-1]), int(order[100])])
+    # shortest, longest and 14 spread over the length order
+    seqs = sorted({int(order[0]), int(order[-1])} | {int(order[i]) for i in range(9, 256, 18)})
+    assert len(seqs) >= 16
     kp, vp, bt, seqs = w.compact_host_pool(seqs)
     B = w.batch
     steps = w.decode_steps                       # all 64; the oracle checks steps 0, 31 and 63
@@ -95,7 +93,7 @@ def test_cfg5_full_decode_steps_sampled():
         assert int(dw.status.item()) == 0
         o, lse = orc.decode_attention(q_rot, kp, vp, bt, ctx, w.num_q_heads)
         H.assert_attn_close(H.torch_to_bits(out)[seqs], o, f"cfg5 full decode step {step}")
-        assert np.abs(lse_d.cpu().numpy()[seqs] - lse).max() <= H.LSE_TOL
+        H.assert_lse_close(lse_d.cpu().numpy()[seqs], lse, "decode")
         assert torch.isfinite(out.float()).all()
         # the fused step on the same inputs (it stores the same k/v again): identical bits at full size
         out_f = torch.empty_like(out)

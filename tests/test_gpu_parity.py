@@ -53,7 +53,7 @@ def _check_turn(w, seqs=None, interleaved=False, use_rope=True, sm_scale=None):
     got_o = H.torch_to_bits(dw.out)[ref["rows"]]
     H.assert_attn_close(got_o, ref["o"], f"{w.name} append-prefill")
     got_lse = dw.lse.cpu().numpy()[ref["rows"]]
-    assert np.abs(got_lse - ref["lse"]).max(initial=0) <= H.LSE_TOL
+    H.assert_lse_close(got_lse, ref["lse"], f"{w.name} append-prefill")
     return dw, ref
 
 
@@ -86,7 +86,7 @@ def test_cfg1_turn_and_decode_steps():
         assert int(dw.status.item()) == 0
         H.assert_rope_close(H.torch_to_bits(dq), q_rot, "decode q")
         H.assert_attn_close(H.torch_to_bits(out), o, f"cfg1 decode step {step}")
-        assert np.abs(lse_d.cpu().numpy() - lse).max() <= H.LSE_TOL
+        H.assert_lse_close(lse_d.cpu().numpy(), lse, "decode")
     pg = w.pages_of(0)
     assert np.array_equal(dw.pages_from_device("v", pg), vp[bt[0, :len(pg)]])
 
@@ -157,7 +157,7 @@ def test_decode_loop_small(name):
         torch.cuda.synchronize()
         assert int(dw.status.item()) == 0
         H.assert_attn_close(H.torch_to_bits(out), o, f"{name} decode step {step}")
-        assert np.abs(lse_d.cpu().numpy() - lse).max() <= H.LSE_TOL
+        H.assert_lse_close(lse_d.cpu().numpy(), lse, "decode")
 
 
 def test_decode_one_long_row_many_chunks():
@@ -189,7 +189,7 @@ def test_decode_one_long_row_many_chunks():
         torch.cuda.synchronize()
         assert int(dw.status.item()) == 0
         H.assert_attn_close(H.torch_to_bits(out), o, f"long row, step {step}")
-        assert np.abs(lse_d.cpu().numpy() - lse).max() <= H.LSE_TOL
+        H.assert_lse_close(lse_d.cpu().numpy(), lse, "decode")
 
 
 def test_decode_zero_length_and_bad_page_flag():
