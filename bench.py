@@ -2,8 +2,8 @@
 """Benchmark of the EFIM per-turn GPU path on synthetic multi-turn infilling batches.
 
 One "step" = one turn of one layer over one ragged batch:
-    efim_kv_append(k, v of the inc tokens; q is not rewritten)
-    -> efim_append_prefill_step (attention; q rotated as it is loaded; planned once per batch)
+    efim_kv_append(inc tokens: q and k rotated, k/v stored in the pages)
+    -> efim_append_prefill_attn_planned (the work list is planned once per batch)
     -> efim_decode_step (kv_append of 1 generated token per sequence fused with decode attention)
 `value` = new tokens (inc + generated) that went through the path per second, inputs
 resident in HBM; `e2e` = the same with the step's q/k/v coming from pinned host
@@ -89,8 +89,6 @@ def workload_counts(w):
         "prefill_kv_bytes": int(4 * D * Hkv * L[has_new].sum()),
         "decode_kv_bytes": int(4 * D * Hkv * (L + 1).sum()) if w.decode_steps > 0 else 0,
         "kv_append_bytes_per_token": 4 * D * (Hq + 2 * Hkv),
-        # what the append moves when q is rotated by the attention kernel instead (k, v read + written)
-        "kv_only_append_bytes_per_token": 4 * D * 2 * Hkv,
     }
 
 
@@ -372,7 +370,8 @@ class TurnRunner:
         self.status = torch.zeros(1, dtype=torch.int32, device=dev)
         self.bits = w.new_qkv()
         self.T = self.bits[0].shape[0]
-        self.q, self.k_new, self.v_new = (self.to_dev(x) for x in self.bits)
+        self.q0, self.k_new, self.v_new = (self.to_dev(x) for x in self.bits)
+        self.q = self.q0.clone()                 # rotated in place by every step, restored between steps
         self.out = torch.empty_like(self.q)
         self.ws_p = torch.empty(max(efim.efim_prefill_workspace_bytes(self.cache, self.batch), 256),
                                 dtype=torch.uint8, device=dev)
@@ -387,7 +386,7 @@ class TurnRunner:
             self.plan_ms = (time.perf_counter() - t_plan) / 10 * 1e3
         if self.has_decode:
             self.dbits = w.decode_qkv(0)
-            self.dq, self.dk, self.dv = (self.to_dev(x) for x in self.dbits)
+            self.dq, self.dk, self.dv = (self.to_dev(x) for x in self.dbits)     # read only (rotated on load)
             self.dout = torch.empty_like(self.dq)
             self.d_ctx = torch.from_numpy(self.ctx_after + 1).to(dev)
             self.max_ctx = int(self.ctx_after.max()) + w.decode_steps
@@ -415,12 +414,11 @@ class TurnRunner:
             *((self.dq, self.dk, self.dv, self.dout) if self.has_decode else (None,) * 4))
         if marks: marks[0].record(self.stream)
         if self.T > 0:
-            efim.efim_kv_append(self.cache, self.batch, self.rope, None, k_, v_, self.status)     # k, v only
+            efim.efim_kv_append(self.cache, self.batch, self.rope, q_, k_, v_, self.status)
         if marks: marks[1].record(self.stream)
         if self.T > 0:
-            # attention; the query rows are rotated as the kernel loads them (k/v = None: appended above)
-            efim.efim_append_prefill_step(self.cache, self.batch, self.rope, q_, None, None, out_, None, 0.0,
-                                          self.ws_p, self.status, plan=self.plan, lists_resident=self.uploaded)
+            efim.efim_append_prefill_attn(self.cache, self.batch, q_, out_, None, 0.0, self.ws_p, self.status,
+                                          plan=self.plan, lists_resident=self.uploaded)
             self.uploaded = True                 # the lists stay at the head of ws_p: uploaded once per batch
         if marks: marks[2].record(self.stream)
         if self.has_decode:
@@ -428,6 +426,13 @@ class TurnRunner:
             efim.efim_decode_step(self.cache, self.w.batch, self.d_ctx, self.max_ctx, self.batch.d_block_table,
                                   self.rope, dq_, dk_, dv_, dout_, None, 0.0, self.ws_d, self.status)
         if marks: marks[3].record(self.stream)
+
+    def restore(self, flush):
+        """Between timed steps, outside the event pairs: the unrotated q back, L2 evicted."""
+        if self.T > 0:
+            self.q.copy_(self.q0)
+        if flush is not None:
+            flush.fill_(1)
 
     def check_status(self):
         st = int(self.status.item())
@@ -445,10 +450,10 @@ def call_records(cnt, seg_ms, peaks, has_decode, decode_tokens=None):
     hbm, tc = peaks["hbm_gbs"], peaks["bf16_tflops"]
     rec = {}
     if cnt["new_tokens"] > 0:
-        app_bytes = cnt["kv_only_append_bytes_per_token"] * cnt["new_tokens"]
+        app_bytes = cnt["kv_append_bytes_per_token"] * cnt["new_tokens"]
         rec["kv_append"] = {"ms": t_app, "bytes": app_bytes, "bound": "hbm", "unit": "GB/s",
                             **frac_pair(app_bytes / t_app / 1e6, hbm, NOMINAL["hbm_gbs"]),
-                            "note": "k and v only (read + page write); q is rotated by the attention kernel"}
+                            "note": "q read + rewritten in place, k and v read + written into the pages"}
         intensity = cnt["prefill_flops"] / max(cnt["prefill_kv_bytes"], 1)
         tflops = cnt["prefill_flops"] / t_pre / 1e9
         ceil_meas = min(tc, intensity * hbm / 1e3)
@@ -460,6 +465,7 @@ def call_records(cnt, seg_ms, peaks, has_decode, decode_tokens=None):
             "ceiling_tflops_measured": ceil_meas, "ceiling_tflops_nominal": ceil_nom,
             "frac_of_measured": tflops / ceil_meas, "frac_of_nominal": tflops / ceil_nom,
             "frac_of_measured_tensor_peak": tflops / tc, "frac_of_nominal_tensor_peak": tflops / NOMINAL["bf16_tflops"],
+            "frac_of_measured_sustained_tensor_peak": tflops / peaks.get("bf16_tflops_sustained", tc),
             "note": "ceiling = min(tensor peak, intensity x HBM bandwidth)"}
     if has_decode:
         rec["decode_step"] = {"ms": t_dec, "bytes": cnt["decode_kv_bytes"], "bound": "hbm", "unit": "GB/s",
@@ -473,15 +479,13 @@ def time_steps(torch, runner, flush, reps, warmup):
     def ev():
         return torch.cuda.Event(enable_timing=True)
     for _ in range(warmup):
-        if flush is not None:
-            flush.fill_(1)
+        runner.restore(flush)
         runner.step()
     torch.cuda.synchronize()
     marks = [[ev() for _ in range(4)] for _ in range(reps)]
     t0 = time.time()
     for i in range(reps):
-        if flush is not None:
-            flush.fill_(1)                     # evict L2 between timed steps (outside the event pairs)
+        runner.restore(flush)                  # evict L2 between timed steps (outside the event pairs)
         runner.step(marks[i])
     torch.cuda.synchronize()
     t1 = time.time()
@@ -665,14 +669,14 @@ def run_native(args):
     # ---------------- device-resident timing: W warm-up steps, then exactly K timed steps
     warm = max(args.warmup, 3)
     for _ in range(warm):
-        flush.fill_(1)
+        r.restore(flush)
         r.step()
     barrier()
     sampler.wait_first()
     marks = [[ev() for _ in range(4)] for _ in range(args.steps)]
     wall0 = time.time()
     for i in range(args.steps):
-        flush.fill_(1)                         # evict L2 between timed steps (outside the event pairs)
+        r.restore(flush)                       # evict L2 between timed steps (outside the event pairs)
         r.step(marks[i])
     barrier()
     wall1 = time.time()
@@ -709,16 +713,16 @@ def run_native(args):
         "append_prefill_kv_gbs": calls["append_prefill"]["kv_gbs"] if "append_prefill" in calls else None,
         "decode_ms": t_dec, "decode_fused_append": True,
         "decode_kv_gbs": calls["decode_step"]["achieved"] if has_decode else None,
-        "q_rotated_by": "the attention kernels, on load (efim_append_prefill_step / efim_decode_step)",
+        "q_rotated_by": "efim_kv_append in place (prefill), the decode kernel on load (efim_decode_step)",
     }
     # dominant call of the step and the roofline that bounds it on this workload
     if t_pre >= t_dec:
         ap = calls["append_prefill"]
         if ap["bound"] == "tensor":
-            roof = {"kernel": "efim_append_prefill_step", "bound": "tensor", "achieved": ap["tflops"],
+            roof = {"kernel": "efim_append_prefill_attn", "bound": "tensor", "achieved": ap["tflops"],
                     "peak": peaks["bf16_tflops"], "unit": "TFLOP/s", "algorithmic": cnt["prefill_flops"]}
         else:
-            roof = {"kernel": "efim_append_prefill_step", "bound": "hbm", "achieved": ap["kv_gbs"],
+            roof = {"kernel": "efim_append_prefill_attn", "bound": "hbm", "achieved": ap["kv_gbs"],
                     "peak": peaks["hbm_gbs"], "unit": "GB/s", "algorithmic": cnt["prefill_kv_bytes"]}
         roof["intensity_flop_per_byte"] = ap["intensity_flop_per_byte"]
     else:

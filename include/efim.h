@@ -363,6 +363,24 @@ void efim_frontend_stats(const efim_frontend* fe, int64_t* h_out);
 int64_t efim_fragment_cuts(uint64_t seed, int64_t n, int32_t lo, int32_t hi, int64_t* h_cuts, int64_t capacity);
 efim_status efim_fim_split(uint64_t seed, int64_t n, int64_t* a, int64_t* b);
 
+/*
+ * One FIM training example with fragment tokenisation (Sec. 2.1 for the PSM layout
+ * `<P>prefix<S>suffix<M>middle`, Sec. 3.2 for the segments): the document of n characters is
+ * split by efim_fim_split(seed), each of the three parts is cut into segments on its own (a
+ * segment never spans a special token; generator seeds seed+1 prefix, seed+2 suffix, seed+3
+ * middle), and the example is the list of spans in the order they are emitted.  h_spans
+ * receives up to `capacity` triples (kind, begin, end): kind EFIM_SPAN_TEXT = tokenise
+ * characters [begin, end) of the document on their own; EFIM_SPAN_TOKEN_P/_S/_M = emit that
+ * special token (begin = end = where the part starts).  Returns the number of spans (call
+ * with capacity 0 to size), -1 for invalid arguments.
+ */
+#define EFIM_SPAN_TEXT     0
+#define EFIM_SPAN_TOKEN_P  1
+#define EFIM_SPAN_TOKEN_S  2
+#define EFIM_SPAN_TOKEN_M  3
+int64_t efim_fim_fragment_spans(uint64_t seed, int64_t n, int32_t lo, int32_t hi, int64_t* h_spans,
+                                int64_t capacity);
+
 #ifdef __cplusplus
 }
 #endif

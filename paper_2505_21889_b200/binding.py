@@ -41,7 +41,7 @@ EXPORTS = ("efim_last_cuda_error", "efim_strerror", "efim_version", "efim_rope_t
            "efim_prefill_launch_count", "efim_decode_launch_count",
            "efim_prefill_plan_bytes", "efim_prefill_plan", "efim_append_prefill_attn_planned", "efim_decode_step",
            "efim_append_prefill_step", "efim_selftest_bounded_wait",
-           "efim_fragment_cuts", "efim_fim_split",
+           "efim_fragment_cuts", "efim_fim_split", "efim_fim_fragment_spans",
            "efim_frontend_create", "efim_frontend_destroy", "efim_frontend_transform", "efim_frontend_admit",
            "efim_frontend_finish", "efim_frontend_stats")
 

@@ -37,3 +37,36 @@ extern "C" efim_status efim_fim_split(uint64_t seed, int64_t n, int64_t* a, int6
   *b = y;
   return EFIM_OK;
 }
+
+// The spans of one training example, in emission order.  A text span is one segment of one of
+// the three parts; the special tokens sit between the parts: <P> prefix.. <S> suffix.. <M> middle..
+extern "C" int64_t efim_fim_fragment_spans(uint64_t seed, int64_t n, int32_t lo, int32_t hi, int64_t* h_spans,
+                                           int64_t capacity) {
+  if (n < 0 || lo < 1 || hi < lo || capacity < 0 || (capacity > 0 && !h_spans)) return -1;
+  int64_t a = 0, b = 0;
+  if (efim_fim_split(seed, n, &a, &b) != EFIM_OK) return -1;
+  const uint64_t span = (uint64_t)(hi - lo) + 1;
+  int64_t count = 0;
+  auto emit = [&](int64_t kind, int64_t begin, int64_t end) {
+    if (count < capacity) {
+      h_spans[3 * count] = kind;
+      h_spans[3 * count + 1] = begin;
+      h_spans[3 * count + 2] = end;
+    }
+    ++count;
+  };
+  // part k is segmented with the generator under seed + 1 + k (prefix, suffix, middle)
+  const int64_t part_begin[3] = {0, b, a}, part_end[3] = {a, n, b};
+  const int64_t marker[3] = {EFIM_SPAN_TOKEN_P, EFIM_SPAN_TOKEN_S, EFIM_SPAN_TOKEN_M};
+  for (int k = 0; k < 3; ++k) {
+    emit(marker[k], part_begin[k], part_begin[k]);
+    int64_t pos = part_begin[k];
+    for (uint64_t i = 0; pos < part_end[k]; ++i) {
+      const int64_t len = lo + (int64_t)(splitmix64(seed + 1 + (uint64_t)k, i) % span);
+      const int64_t next = (part_end[k] - pos <= len) ? part_end[k] : pos + len;
+      emit(EFIM_SPAN_TEXT, pos, next);
+      pos = next;
+    }
+  }
+  return count;
+}

@@ -86,3 +86,52 @@ def test_library_example_equals_oracle_and_rejects_bad_ranges():
     for bad in [(-1, 1, 200), (10, 0, 200), (10, 5, 4)]:
         with pytest.raises(EfimError):
             fr.segment_cuts(1, *bad)
+
+
+def test_library_spans_are_the_psm_layout():
+    """The span list itself, against facts that need no oracle: markers in the order P, S, M;
+    the text spans between them tile prefix [0,a), suffix [b,n), middle [a,b) without gaps;
+    every segment but a part's last is within [lo, hi]."""
+    n, lo, hi = 5000, 3, 40
+    spans = fr.fim_fragment_spans(5, n, lo, hi).tolist()
+    a, b = fr.fim_split(5, n)
+    kinds = [k for k, _, _ in spans if k != 0]
+    assert kinds == [1, 2, 3]
+    parts, cur = [], None
+    for kind, begin, end in spans:
+        if kind != 0:
+            cur = []
+            parts.append(cur)
+            assert begin == end
+        else:
+            cur.append((begin, end))
+    for part, (pb, pe) in zip(parts, [(0, a), (b, n), (a, b)]):
+        pos = pb
+        for i, (begin, end) in enumerate(part):
+            assert begin == pos and end > begin
+            assert end - begin <= hi and (i == len(part) - 1 or end - begin >= lo)
+            pos = end
+        assert pos == pe
+
+
+def test_command_emits_fragment_tokenised_examples(tmp_path, capsys):
+    import json
+    doc = "def complete(self):\n    return self.models\n" * 30
+    f1, f2 = tmp_path / "a.py", tmp_path / "b.py"
+    f1.write_text(doc)
+    f2.write_text(doc[::-1])
+    assert fr.main([str(f1), str(f2), "--seed", "3", "--hi", "50", "--tokenizer", "chars",
+                    "--special", "70001", "70002", "70003"]) == 0
+    lines = [json.loads(ln) for ln in capsys.readouterr().out.splitlines()]
+    assert [ln["seed"] for ln in lines] == [3, 7] and lines[0]["chars"] == len(doc)
+    for ln, text in zip(lines, (doc, doc[::-1])):
+        want = fo.fim_fragment_example(text, lambda seg: [ord(c) for c in seg], ln["seed"], 70001, 70002, 70003, 1, 50)
+        assert ln["input_ids"] == want
+        ids = ln["input_ids"]
+        s_at, m_at = ids.index(70002), ids.index(70003)
+        back = lambda xs: "".join(chr(t) for t in xs)
+        assert back(ids[1:s_at]) + back(ids[m_at + 1:]) + back(ids[s_at + 1:m_at]) == text   # prefix+middle+suffix
+    # the default tokenizer: UTF-8 bytes
+    assert fr.main([str(f1), "--seed", "1"]) == 0
+    out = json.loads(capsys.readouterr().out)
+    assert max(out["input_ids"]) <= 258 and out["segments"] >= 3
