@@ -45,7 +45,11 @@ __device__ __forceinline__ void transposed_reduce(float* x, int j) {
 // the ring 64 KB per CTA at D = 128, so three CTAs (12 warps) share an SM: the kernel is
 // short of warps to issue from, not of bytes in flight (with three stages and two CTAs
 // per SM it ran at 84 % of the measured copy bandwidth, with two and three at 99 %).
-constexpr int DEC_STAGES = 2;
+// Group tiles of more than 4 query heads need the registers of a third CTA for their q and o
+// rows: they run two CTAs to an SM and take a third stage instead.
+constexpr int DEC_MAX_STAGES = 3;
+__host__ __device__ constexpr int dec_stages(int group_tile) { return group_tile > 4 ? 3 : 2; }
+__host__ __device__ constexpr int dec_ctas_per_sm(int group_tile) { return group_tile > 4 ? 2 : 3; }
 
 __device__ __forceinline__ void dec_bulk_load(uint32_t dst, const void* src, uint32_t bytes, uint32_t bar) {
   asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];" ::"r"(dst),
@@ -86,16 +90,22 @@ __device__ __forceinline__ uint4 dec_rotate_vec(uint4 mine, uint4 other, const f
   return mine;
 }
 
+// GT query heads of one kv head per CTA.  Up to 4 heads are scored in one pass over a staged
+// page; 5 to 7 in two passes of 4 (the second padded with zero queries) over the same page in
+// shared memory - the K/V bytes come from HBM once.
 template <int D, int GT, bool FUSED>
-__global__ void __launch_bounds__(128, 3) decode_splitkv_kernel(const DecodeParams p) {
+__global__ void __launch_bounds__(128, dec_ctas_per_sm(GT)) decode_splitkv_kernel(const DecodeParams p) {
+  constexpr int DEC_STAGES = dec_stages(GT);
   constexpr int LPT = D / 8;            // lanes sharing one token row
   constexpr int TPS = 32 / LPT;         // tokens per warp-wide 16-byte read
   constexpr int STEPS = 16 / TPS;       // reads per page
-  constexpr int GP = (GT + 1) & ~1;     // heads padded to even
-  constexpr int NV = STEPS * GP;        // partial dot products per lane per page
-  constexpr int NF = GP / 2;            // finished scores per lane per page
+  constexpr int PH = GT > 4 ? 2 : 1;    // passes over a page's keys
+  constexpr int HPP = GT > 4 ? 4 : ((GT + 1) & ~1);   // heads per pass (padded to even)
+  constexpr int GP = PH * HPP;          // heads with padding
+  constexpr int NV = STEPS * HPP;       // partial dot products per lane per pass
+  constexpr int NF = HPP / 2;           // finished scores per lane per pass
   constexpr int PAGE_BYTES = 16 * D * 2;
-  static_assert(NV / LPT == NF, "reduction leaves GP/2 values per lane");
+  static_assert(NV / LPT == NF, "reduction leaves HPP/2 values per lane");
 
   extern __shared__ __align__(128) uint8_t dec_ring[];   // [4 warps][DEC_STAGES][K page | V page]
   __shared__ __align__(8) uint64_t s_bar[4][DEC_STAGES];
@@ -202,9 +212,9 @@ __global__ void __launch_bounds__(128, 3) decode_splitkv_kernel(const DecodePara
 
   // q and o as packed fp32 pairs (dims 2e, 2e+1): the inner products and the P V
   // update run on two-wide FMAs
-  uint64_t q2[GT][4];
+  uint64_t q2[GP][4];
 #pragma unroll
-  for (int g = 0; g < GT; ++g) {
+  for (int g = 0; g < GP; ++g) {
     if (g < ng) {
       const uint4* qrow = reinterpret_cast<const uint4*>(p.q + ((size_t)r * p.Hq + head0 + g) * D);
       uint4 w = __ldg(qrow + j);
@@ -222,11 +232,13 @@ __global__ void __launch_bounds__(128, 3) decode_splitkv_kernel(const DecodePara
   for (int g = 0; g < GT; ++g)
 #pragma unroll
     for (int e = 0; e < 4; ++e) o2[g][e] = 0ull;
-  float m_run[GP], l_part[NF];
+  float m_run[GP], l_part[PH][NF];
 #pragma unroll
   for (int g = 0; g < GP; ++g) m_run[g] = -INFINITY;
 #pragma unroll
-  for (int i = 0; i < NF; ++i) l_part[i] = 0.f;
+  for (int ph = 0; ph < PH; ++ph)
+#pragma unroll
+    for (int i = 0; i < NF; ++i) l_part[ph][i] = 0.f;
 
   const int odd = j & 1;
   const int st_mine = j >> 1;                   // step whose scores this lane ends up with
@@ -272,59 +284,65 @@ __global__ void __launch_bounds__(128, 3) decode_splitkv_kernel(const DecodePara
     if (page_ok) {
       const uint8_t* kst = ring + sg * 2 * PAGE_BYTES + (tg * D + j * 8) * 2;
       const uint8_t* vst = kst + PAGE_BYTES;
-      // ---- scores: partial dot products over this lane's 8 dims, then the cross-lane sum
-      float x[NV];
-#pragma unroll
-      for (int st = 0; st < STEPS; ++st) {
-        const uint4 kv = *reinterpret_cast<const uint4*>(kst + st * TPS * D * 2);
-        const uint32_t* u = reinterpret_cast<const uint32_t*>(&kv);
-        uint64_t k2[4];
-#pragma unroll
-        for (int e = 0; e < 4; ++e) k2[e] = pack2(bf16lo(u[e]), bf16hi(u[e]));
-#pragma unroll
-        for (int g = 0; g < GP; ++g) {
-          float acc = 0.f;
-          if (g < GT) {
-            uint64_t a2 = 0ull;
-#pragma unroll
-            for (int e = 0; e < 4; ++e) a2 = ffma2(q2[g][e], k2[e], a2);
-            float lo, hi;
-            unpack2(a2, lo, hi);
-            acc = lo + hi;
-          }
-          x[st * GP + g] = acc;
-        }
-      }
-      transposed_reduce<NV, LPT>(x, j);
-      // lane j now holds, for token (st_mine*TPS + tg) of the page, heads odd*NF + i
-      const int tok_in_page = st_mine * TPS + tg;
+      // ---- scores: partial dot products over this lane's 8 dims, then the cross-lane sum;
+      // HPP heads per pass
+      const int tok_in_page = st_mine * TPS + tg;       // the token whose scores this lane ends up with
       const bool visible = (pg << 4) + tok_in_page < end;
-      float sc[NF], mx[NF];
+      float alpha[GP];
 #pragma unroll
-      for (int a = 0; a < NF; ++a) { sc[a] = visible ? x[a] : -INFINITY; mx[a] = sc[a]; }
+      for (int ph = 0; ph < PH; ++ph) {
+        float x[NV];
 #pragma unroll
-      for (int off = 2; off < 32; off <<= 1)
+        for (int st = 0; st < STEPS; ++st) {
+          const uint4 kv = *reinterpret_cast<const uint4*>(kst + st * TPS * D * 2);
+          const uint32_t* u = reinterpret_cast<const uint32_t*>(&kv);
+          uint64_t k2[4];
 #pragma unroll
-        for (int a = 0; a < NF; ++a) mx[a] = fmaxf(mx[a], __shfl_xor_sync(0xffffffffu, mx[a], off));
-      float alpha[GP], mine[NF], alpha_mine[NF];
+          for (int e = 0; e < 4; ++e) k2[e] = pack2(bf16lo(u[e]), bf16hi(u[e]));
 #pragma unroll
-      for (int a = 0; a < NF; ++a) {
-        const float other = __shfl_xor_sync(0xffffffffu, mx[a], 1);
-        const float m_lo = odd ? other : mx[a];       // head a
-        const float m_hi = odd ? mx[a] : other;       // head NF + a
-        const float n_lo = fmaxf(m_run[a], m_lo), n_hi = fmaxf(m_run[NF + a], m_hi);
-        alpha[a] = exp2f(m_run[a] - n_lo);
-        alpha[NF + a] = exp2f(m_run[NF + a] - n_hi);
-        m_run[a] = n_lo;
-        m_run[NF + a] = n_hi;
-        mine[a] = odd ? n_hi : n_lo;
-        alpha_mine[a] = odd ? alpha[NF + a] : alpha[a];
-      }
+          for (int g = 0; g < HPP; ++g) {
+            float acc = 0.f;
+            if (ph * HPP + g < GT) {
+              uint64_t a2 = 0ull;
 #pragma unroll
-      for (int a = 0; a < NF; ++a) {
-        const float pr = exp2f(sc[a] - mine[a]);      // masked: exp2(-inf) = 0
-        l_part[a] = fmaf(l_part[a], alpha_mine[a], pr);
-        s_p[warp][tok_in_page][odd * NF + a] = pr;
+              for (int e = 0; e < 4; ++e) a2 = ffma2(q2[ph * HPP + g][e], k2[e], a2);
+              float lo, hi;
+              unpack2(a2, lo, hi);
+              acc = lo + hi;
+            }
+            x[st * HPP + g] = acc;
+          }
+        }
+        transposed_reduce<NV, LPT>(x, j);
+        // lane j now holds, for token (st_mine*TPS + tg) of the page, heads ph*HPP + odd*NF + i
+        float sc[NF], mx[NF];
+#pragma unroll
+        for (int a = 0; a < NF; ++a) { sc[a] = visible ? x[a] : -INFINITY; mx[a] = sc[a]; }
+#pragma unroll
+        for (int off = 2; off < 32; off <<= 1)
+#pragma unroll
+          for (int a = 0; a < NF; ++a) mx[a] = fmaxf(mx[a], __shfl_xor_sync(0xffffffffu, mx[a], off));
+        float mine[NF], alpha_mine[NF];
+#pragma unroll
+        for (int a = 0; a < NF; ++a) {
+          const int h_lo = ph * HPP + a, h_hi = ph * HPP + NF + a;
+          const float other = __shfl_xor_sync(0xffffffffu, mx[a], 1);
+          const float m_lo = odd ? other : mx[a];       // head h_lo
+          const float m_hi = odd ? mx[a] : other;       // head h_hi
+          const float n_lo = fmaxf(m_run[h_lo], m_lo), n_hi = fmaxf(m_run[h_hi], m_hi);
+          alpha[h_lo] = exp2f(m_run[h_lo] - n_lo);
+          alpha[h_hi] = exp2f(m_run[h_hi] - n_hi);
+          m_run[h_lo] = n_lo;
+          m_run[h_hi] = n_hi;
+          mine[a] = odd ? n_hi : n_lo;
+          alpha_mine[a] = odd ? alpha[h_hi] : alpha[h_lo];
+        }
+#pragma unroll
+        for (int a = 0; a < NF; ++a) {
+          const float pr = exp2f(sc[a] - mine[a]);      // masked: exp2(-inf) = 0
+          l_part[ph][a] = fmaf(l_part[ph][a], alpha_mine[a], pr);
+          s_p[warp][tok_in_page][ph * HPP + odd * NF + a] = pr;
+        }
       }
       __syncwarp();
       // ---- values
@@ -384,10 +402,14 @@ __global__ void __launch_bounds__(128, 3) decode_splitkv_kernel(const DecodePara
 #pragma unroll
   for (int off = 2; off < 32; off <<= 1)
 #pragma unroll
-    for (int i = 0; i < NF; ++i) l_part[i] += __shfl_xor_sync(0xffffffffu, l_part[i], off);
+    for (int ph = 0; ph < PH; ++ph)
+#pragma unroll
+      for (int i = 0; i < NF; ++i) l_part[ph][i] += __shfl_xor_sync(0xffffffffu, l_part[ph][i], off);
   if (lane < 2) {
 #pragma unroll
-    for (int i = 0; i < NF; ++i) s_l[warp][lane * NF + i] = l_part[i];
+    for (int ph = 0; ph < PH; ++ph)
+#pragma unroll
+      for (int i = 0; i < NF; ++i) s_l[warp][ph * HPP + lane * NF + i] = l_part[ph][i];
   }
   if (lane == 0) {
 #pragma unroll
@@ -492,8 +514,16 @@ __global__ void __launch_bounds__(128) decode_merge_kernel(const DecodeParams p)
 DecodePlan plan_decode(int rows, int Hq, int Hkv, int D, int max_len) {
   DecodePlan pl;
   const int G = Hq / Hkv;
-  pl.group_tile = G >= 4 ? 4 : G;
-  if (G % 4 != 0 && G > 4) pl.group_tile = (G % 3 == 0) ? 3 : 4;
+  // Groups of up to 7 query heads share one CTA's walk over the K/V pages (5 to 7 in two
+  // passes over the page in shared memory: 3.1-3.7 TB/s of K/V against 3.0 when the pages
+  // were fetched twice).  From 8 heads on the fp32 FMAs, not the bytes, are the bound (8 heads
+  // in one CTA measured 1.9 TB/s against 3.2 as two CTAs of 4), so larger groups are cut into
+  // tiles of 4, or of 3 where that divides the group and 4 does not.
+  if (G <= 7) {
+    pl.group_tile = G;
+  } else {
+    pl.group_tile = (G % 4 != 0 && G % 3 == 0) ? 3 : 4;
+  }
   pl.gsplit = (G + pl.group_tile - 1) / pl.group_tile;
   if (max_len < 1) max_len = 1;
   // Aim for ~32 CTAs per SM over the launch so that ragged lengths even out, but keep a
@@ -523,7 +553,7 @@ DecodePlan plan_decode(int rows, int Hq, int Hkv, int D, int max_len) {
 
 template <int D, int GT, bool FUSED>
 static efim_status launch_split_f(const DecodeParams& p, dim3 grid, cudaStream_t s) {
-  constexpr int ring_bytes = 4 * DEC_STAGES * 2 * 16 * D * 2;      // 4 warps x stages x (K page + V page)
+  constexpr int ring_bytes = 4 * dec_stages(GT) * 2 * 16 * D * 2;  // 4 warps x stages x (K page + V page)
   EFIM_CUDA_TRY(cudaFuncSetAttribute(decode_splitkv_kernel<D, GT, FUSED>,
                                      cudaFuncAttributeMaxDynamicSharedMemorySize, ring_bytes));
   decode_splitkv_kernel<D, GT, FUSED><<<grid, 128, ring_bytes, s>>>(p);
@@ -542,7 +572,10 @@ static efim_status launch_decode_d(const DecodeParams& p, const DecodePlan& pl, 
     case 1: st = launch_split<D, 1>(p, grid, s); break;
     case 2: st = launch_split<D, 2>(p, grid, s); break;
     case 3: st = launch_split<D, 3>(p, grid, s); break;
-    default: st = launch_split<D, 4>(p, grid, s); break;
+    case 4: st = launch_split<D, 4>(p, grid, s); break;
+    case 5: st = launch_split<D, 5>(p, grid, s); break;
+    case 6: st = launch_split<D, 6>(p, grid, s); break;
+    default: st = launch_split<D, 7>(p, grid, s); break;
   }
   if (st != EFIM_OK) return st;
   EFIM_CUDA_TRY(cudaGetLastError());

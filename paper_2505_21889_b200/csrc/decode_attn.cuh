@@ -34,7 +34,7 @@ struct DecodeParams {
 };
 
 struct DecodePlan {
-  int group_tile;             // q heads of one kv head handled per CTA (<= 4)
+  int group_tile;             // q heads of one kv head handled per CTA (<= 7)
   int gsplit;                 // CTAs per kv head
   int chunk_tokens;           // keys per chunk (multiple of 64)
   int n_chunks;

@@ -222,6 +222,27 @@ def test_step_call_reports_a_position_beyond_the_rotary_table():
     H.assert_attn_close(H.torch_to_bits(dw.out)[ref["rows"]], ref["o"], "the sequence inside the table")
 
 
+def test_many_single_tile_items_beside_long_row_blocks():
+    """More items of at most 128 rows than two per SM, beside row blocks of 256: all rows
+    against the oracle, and the same bits from run to run."""
+    efim, H, _custom, _check_turn = _mods()
+    rng = np.random.default_rng(77)
+    B, Hq = 11, 32
+    cached = rng.integers(0, 700, size=B).astype(np.int32)
+    new = rng.integers(1, 129, size=B).astype(np.int32)
+    new[3], cached[3] = 128, 256                  # a full tile on a tile edge
+    new[5], cached[5] = 300, 90                   # two row blocks: 256 rows and 44 rows
+    new[7], cached[7] = 1, 0                      # a lone first token
+    w = _custom(Hq, Hq, 128, cached, new, seed=31)
+    dw, ref = _check_turn(w)
+    first = (H.torch_to_bits(dw.out).copy(), dw.lse.cpu().numpy().copy())
+    dw.out.zero_()
+    dw.lse.zero_()
+    dw.gpu_prefill()
+    torch.cuda.synchronize()
+    assert np.array_equal(H.torch_to_bits(dw.out), first[0]) and np.array_equal(dw.lse.cpu().numpy(), first[1])
+
+
 def test_bounded_wait_expires_and_reports():
     """One warp waits on a barrier nothing completes, with nothing in flight: after the
     limit the kernel sets EFIM_DEV_TIMEOUT and ends normally; the context stays usable."""

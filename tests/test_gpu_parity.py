@@ -160,6 +160,46 @@ def test_decode_loop_small(name):
         H.assert_lse_close(lse_d.cpu().numpy(), lse, "decode")
 
 
+@pytest.mark.parametrize("Hq,Hkv,D", [(5, 1, 128), (12, 2, 128), (7, 1, 64), (28, 4, 128), (8, 1, 128), (16, 1, 128),
+                                        (20, 2, 64)])
+def test_decode_group_sizes_against_oracle(Hq, Hkv, D):
+    """Groups of 5 to 8 query heads per kv head run in one CTA (two passes over the page in
+    shared memory); larger groups are cut evenly.  Plain and fused steps against the oracle."""
+    H = _harness()
+    import paper_2505_21889_b200 as efim
+    ctx0 = [1, 15, 16, 17, 333, 1200, 2100]
+    w = _custom(Hq, Hkv, D, ctx0, [0] * len(ctx0), seed=Hq * 100 + D, extra=3)
+    dw = H.DeviceWorkload(w)
+    kp, vp, bt, seqs = w.compact_host_pool()
+    ctx = np.array(ctx0, np.int32)
+    B = w.batch
+    max_ctx = int(ctx.max()) + 3
+    ws = torch.empty(max(efim.efim_decode_workspace_bytes(dw.cache, B, max_ctx), 256), dtype=torch.uint8, device="cuda")
+    one = np.ones(B, np.int32)
+    for step in range(3):
+        q, k, v = w.decode_qkv(step)
+        q_rot = orc.kv_append(kp, vp, bt, ctx, one, q, k, v, w.rope_base)
+        ctx = ctx + 1
+        o, lse = orc.decode_attention(q_rot, kp, vp, bt, ctx, Hq)
+        dq, dk, dv = H.bits_to_torch(q), H.bits_to_torch(k), H.bits_to_torch(v)
+        out = torch.empty_like(dq)
+        lse_d = torch.empty((B, Hq), dtype=torch.float32, device="cuda")
+        d_ctx = torch.from_numpy(ctx).cuda()
+        if step == 1:                                  # the two-call form in the middle of the loop
+            efim.efim_kv_append(dw.cache, efim.Batch(ctx - 1, one, dw.batch.d_block_table), dw.rope, dq, dk, dv, dw.status)
+            efim.efim_decode_attn(dw.cache, B, d_ctx, max_ctx, dw.batch.d_block_table, dq, out, lse_d, 0.0, ws, dw.status)
+        else:
+            efim.efim_decode_step(dw.cache, B, d_ctx, max_ctx, dw.batch.d_block_table, dw.rope, dq, dk, dv, out, lse_d,
+                                  0.0, ws, dw.status)
+        torch.cuda.synchronize()
+        assert int(dw.status.item()) == 0
+        H.assert_attn_close(H.torch_to_bits(out), o, f"G={Hq // Hkv} D={D} step {step}")
+        H.assert_lse_close(lse_d.cpu().numpy(), lse, f"G={Hq // Hkv} D={D} step {step}")
+    used = np.array(sorted(set(w.block_table[w.block_table >= 0].tolist())), np.int64)
+    assert np.array_equal(dw.pages_from_device("v", used), vp)
+    H.assert_rope_close(dw.pages_from_device("k", used), kp, "k pages after the loop")
+
+
 def test_decode_one_long_row_many_chunks():
     """A lone long row is cut into more than 32 chunks (so that every SM gets work); the merge
     then takes more than one pass over the lanes for the chunks' lse values."""
@@ -309,10 +349,12 @@ def test_planned_prefill_is_bit_identical_and_checks_its_plan(name):
 
 
 @pytest.mark.parametrize("Hq,Hkv,D,interleaved,use_rope", [
-    (8, 2, 128, False, True),     # group of 4: one CTA per kv head
-    (7, 1, 128, False, True),     # group of 7: two CTAs share the new token's page
+    (8, 2, 128, False, True),     # group of 4: one pass over a page's keys
+    (7, 1, 128, False, True),     # group of 7: two passes over the staged page, K/V fetched once
     (4, 4, 64, True, True),       # head_dim 64, interleaved pairing
     (6, 2, 64, False, False),     # no rotation
+    (10, 2, 128, True, True),     # group of 5
+    (16, 1, 64, False, True),     # group of 16: two CTAs of 8 heads share the new token's page
 ])
 def test_fused_decode_step_equals_append_then_decode(Hq, Hkv, D, interleaved, use_rope):
     """efim_decode_step against efim_kv_append + efim_decode_attn on the same inputs, over
