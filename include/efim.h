@@ -18,8 +18,10 @@
  *     owns all memory and the stream; the library allocates no device memory and never
  *     synchronises the device.  What it keeps between calls: the fixed array of
  *     efim_decode_attn_static (and its per-device address), the SM count of each device it
- *     has planned for, and the driver entry point it encodes tensor maps with - host-side
- *     look-ups made once; no call's result depends on an earlier call.
+ *     has planned for, the driver entry point it encodes tensor maps with, the encoded maps
+ *     of the pools each host thread used last and which devices have had a kernel's
+ *     shared-memory limit raised - host-side look-ups made once; no call's result depends
+ *     on an earlier call.
  *   - `stream` is a cudaStream_t passed as void* (NULL = default stream).  All
  *     work is enqueued on it; results are ready when the stream reaches that point.
  *   - Stream capture: calls that copy a work list from pageable host memory must not be

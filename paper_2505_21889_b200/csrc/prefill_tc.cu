@@ -19,6 +19,7 @@
 #include <vector>
 #include <algorithm>
 #include <functional>
+#include <atomic>
 
 namespace efim {
 namespace pf {
@@ -851,15 +852,53 @@ static bool make_pool_map(CUtensorMap* m, void* pool, int pages, int Hkv, int D)
             CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
+// A model calls this once per layer with the same few pools over and over: the encoded maps
+// of the pools seen last are kept per host thread (a map is a pure function of the key).
+struct PoolMapEntry {
+  void* pool;
+  int pages, Hkv, D;
+  CUtensorMap map;
+};
+static const CUtensorMap* pool_map(void* pool, int pages, int Hkv, int D) {
+  constexpr int kEntries = 16;
+  thread_local PoolMapEntry cache[kEntries] = {};
+  thread_local int next = 0;
+  for (int i = 0; i < kEntries; ++i)
+    if (cache[i].pool == pool && cache[i].pages == pages && cache[i].Hkv == Hkv && cache[i].D == D)
+      return &cache[i].map;
+  PoolMapEntry& e = cache[next];
+  next = (next + 1) % kEntries;
+  e.pool = nullptr;
+  if (!make_pool_map(&e.map, pool, pages, Hkv, D)) return nullptr;
+  e.pool = pool;
+  e.pages = pages;
+  e.Hkv = Hkv;
+  e.D = D;
+  return &e.map;
+}
+
+// The kernel's shared-memory size has to be raised once per device.
 template <int D>
-static efim_status launch_d(const efim_cache_desc* c, const Params& p, const Plan& pl, cudaStream_t s) {
-  CUtensorMap mk, mv;
-  if (!make_pool_map(&mk, c->d_k_pool, c->num_pages, c->num_kv_heads, D) ||
-      !make_pool_map(&mv, c->d_v_pool, c->num_pages, c->num_kv_heads, D))
-    return EFIM_ERR_CUDA;
-  // per device and cheap, so set on every launch rather than cached
+static efim_status raise_smem_limit() {
+  constexpr int kMaxDevices = 64;
+  static std::atomic<bool> done[kMaxDevices];
+  int dev = 0;
+  EFIM_CUDA_TRY(cudaGetDevice(&dev));
+  if (dev >= 0 && dev < kMaxDevices && done[dev].load(std::memory_order_acquire)) return EFIM_OK;
   EFIM_CUDA_TRY(cudaFuncSetAttribute(prefill_tc_kernel<D>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                      Smem<D>::TOTAL));
+  if (dev >= 0 && dev < kMaxDevices) done[dev].store(true, std::memory_order_release);
+  return EFIM_OK;
+}
+
+template <int D>
+static efim_status launch_d(const efim_cache_desc* c, const Params& p, const Plan& pl, cudaStream_t s) {
+  const CUtensorMap* pk = pool_map(c->d_k_pool, c->num_pages, c->num_kv_heads, D);
+  const CUtensorMap* pv = pool_map(c->d_v_pool, c->num_pages, c->num_kv_heads, D);
+  if (!pk || !pv) return EFIM_ERR_CUDA;
+  const CUtensorMap mk = *pk, mv = *pv;
+  const efim_status st = raise_smem_limit<D>();
+  if (st != EFIM_OK) return st;
   prefill_tc_kernel<D><<<pl.n_items, THREADS, Smem<D>::TOTAL, s>>>(p, mk, mv);
   EFIM_CUDA_TRY(cudaGetLastError());
   if (pl.s_max > 1) {

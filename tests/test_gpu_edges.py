@@ -243,6 +243,91 @@ def test_many_single_tile_items_beside_long_row_blocks():
     assert np.array_equal(H.torch_to_bits(dw.out), first[0]) and np.array_equal(dw.lse.cpu().numpy(), first[1])
 
 
+@pytest.mark.parametrize("Hq,Hkv,D", [(8, 2, 128), (4, 4, 64), (7, 1, 128)])
+def test_decode_rows_of_very_different_lengths_in_a_few_chunks(Hq, Hkv, D):
+    """A handful of chunks per row: rows that end in the first chunk (their later chunks have
+    no keys), an empty row and rows that end on and just past a chunk edge, against the
+    oracle; twice, for run-to-run identity."""
+    efim, H, _custom, _check_turn = _mods()
+    lens = np.array([1, 300, 0, 1500, 700, 1499, 256, 257], np.int32)
+    w = _custom(Hq, Hkv, D, np.maximum(lens, 1), [0] * len(lens), seed=41, extra=0)
+    dw = H.DeviceWorkload(w)
+    B, max_ctx = len(lens), 1500
+    assert efim.efim_decode_launch_count(dw.cache, B, max_ctx) == 2
+    ws = torch.empty(efim.efim_decode_workspace_bytes(dw.cache, B, max_ctx), dtype=torch.uint8, device="cuda")
+    kp, vp, bt, seqs = w.compact_host_pool()
+    q = w._normal_bits(3, (B, Hq, D))
+    o, lse = orc.decode_attention(q, kp, vp, bt, lens, Hq)
+    dq = H.bits_to_torch(q)
+    outs = []
+    for _ in range(2):
+        out = torch.full_like(dq, 9.0)
+        lse_d = torch.full((B, Hq), 9.0, dtype=torch.float32, device="cuda")
+        efim.efim_decode_attn(dw.cache, B, torch.from_numpy(lens).cuda(), max_ctx, dw.batch.d_block_table, dq, out, lse_d,
+                              0.0, ws, dw.status)
+        torch.cuda.synchronize()
+        assert int(dw.status.item()) == 0
+        outs.append((out, lse_d))
+    assert torch.equal(outs[0][0].view(torch.int16), outs[1][0].view(torch.int16)) and torch.equal(outs[0][1], outs[1][1])
+    out, lse_d = outs[0]
+    assert torch.all(out[2] == 0) and torch.all(torch.isinf(lse_d[2]))
+    keep = lens > 0
+    H.assert_attn_close(H.torch_to_bits(out)[keep], o[keep], "decode, ragged rows")
+    H.assert_lse_close(lse_d.cpu().numpy()[keep], lse[keep], "decode, ragged rows")
+
+
+def test_garbage_beyond_the_context_and_odd_cached_values():
+    """What a real cache holds: the slots of a sequence's last page beyond its context are
+    uninitialised (here NaN and Inf patterns, in K and in V), and cached values include
+    zeros of both signs, bf16 subnormals and entries several sigma out.  Neither the prefill
+    nor the decode kernel may let the former leak into a result; the latter must be read
+    exactly (the oracle gets the same bits)."""
+    efim, H, _custom, _check_turn = _mods()
+    w = _custom(8, 2, 128, [300, 77, 130], [40, 3, 129], seed=51, extra=2)
+    odd = np.array([0x0000, 0x8000, 0x0001, 0x807F, 0x0040, 0x4100, 0xC120, 0x3F80], np.uint16)  # 0, -0, subnormals, 8, -10, 1
+    real_page_bits = w.page_bits
+
+    def page_bits(which, page_ids):
+        out = real_page_bits(which, page_ids)
+        flat = out.reshape(len(page_ids), -1)
+        flat[:, 5::97] = odd[(np.arange(flat[:, 5::97].shape[1]) + (0 if which == "k" else 3)) % len(odd)]
+        return out
+    w.page_bits = page_bits
+    dw = H.DeviceWorkload(w)
+    used = np.array(sorted(set(w.block_table[w.block_table >= 0].tolist())), np.int64)
+    idx = torch.as_tensor(used, device="cuda")
+    dw.k_pool[idx] = H.bits_to_torch(page_bits("k", used))
+    dw.v_pool[idx] = H.bits_to_torch(page_bits("v", used))
+    nan_inf = torch.tensor([0x7FC0, 0x7F80, 0xFF80, 0x7FFF], dtype=torch.int32).to(torch.int16).cuda().view(torch.bfloat16)
+    for sq in range(w.batch):
+        L = int(w.cached_len[sq] + w.new_len[sq])
+        pg, slot = int(w.block_table[sq, L // 16]), L % 16       # the page the context ends in, first slot beyond it
+        for pool in (dw.k_pool, dw.v_pool):
+            pool[pg, :, slot:, :] = nan_inf[torch.arange(pool[pg, :, slot:, :].numel(), device="cuda") % 4].view(
+                pool[pg, :, slot:, :].shape)
+    dw.gpu_kv_append()
+    dw.gpu_prefill()
+    torch.cuda.synchronize()
+    assert int(dw.status.item()) == 0
+    ref = dw.oracle_turn()
+    H.assert_attn_close(H.torch_to_bits(dw.out), ref["o"], "prefill beside NaN slots")
+    H.assert_lse_close(dw.lse.cpu().numpy(), ref["lse"], "prefill beside NaN slots")
+    # decode over the same contexts (every key so far; the NaN slots lie just beyond)
+    ctx = (w.cached_len + w.new_len).astype(np.int32)
+    q = w._normal_bits(8, (w.batch, 8, 128))
+    o, lse = orc.decode_attention(q, ref["k_pool"], ref["v_pool"], ref["bt"], ctx, 8)
+    out = torch.empty((w.batch, 8, 128), dtype=torch.bfloat16, device="cuda")
+    lse_d = torch.empty((w.batch, 8), dtype=torch.float32, device="cuda")
+    ws = torch.empty(max(efim.efim_decode_workspace_bytes(dw.cache, w.batch, int(ctx.max())), 256), dtype=torch.uint8,
+                     device="cuda")
+    efim.efim_decode_attn(dw.cache, w.batch, torch.from_numpy(ctx).cuda(), int(ctx.max()), dw.batch.d_block_table,
+                          H.bits_to_torch(q), out, lse_d, 0.0, ws, dw.status)
+    torch.cuda.synchronize()
+    assert int(dw.status.item()) == 0
+    H.assert_attn_close(H.torch_to_bits(out), o, "decode beside NaN slots")
+    H.assert_lse_close(lse_d.cpu().numpy(), lse, "decode beside NaN slots")
+
+
 def test_bounded_wait_expires_and_reports():
     """One warp waits on a barrier nothing completes, with nothing in flight: after the
     limit the kernel sets EFIM_DEV_TIMEOUT and ends normally; the context stays usable."""

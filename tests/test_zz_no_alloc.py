@@ -61,11 +61,11 @@ def test_static_scratch_rejects_oversized_requests():
     import tests.gpu_harness as H
     w = make_workload("cfg5", small=True)
     dw = H.DeviceWorkload(w)
-    rows = 4096                                   # far more (row, head, chunk) partials than 8 MiB holds
-    big_ctx = dw.batch.d_block_table.shape[1] * 16
+    rows, big_ctx = 512, 20000                    # 10 chunks of partials per (row, head): more than 8 MiB holds
+    table = torch.zeros((rows, big_ctx // 16), dtype=torch.int32, device="cuda")
     assert efim.efim_decode_workspace_bytes(dw.cache, rows, big_ctx) > efim.efim_decode_static_scratch_bytes()
     d_ctx = torch.ones(rows, dtype=torch.int32, device="cuda")
     q = torch.zeros((rows, w.num_q_heads, w.head_dim), dtype=torch.bfloat16, device="cuda")
     with pytest.raises(efim.EfimError) as e:
-        efim.efim_decode_attn_static(dw.cache, rows, d_ctx, big_ctx, dw.batch.d_block_table, q, torch.empty_like(q))
+        efim.efim_decode_attn_static(dw.cache, rows, d_ctx, big_ctx, table, q, torch.empty_like(q))
     assert e.value.code == 4
