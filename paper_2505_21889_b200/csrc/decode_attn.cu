@@ -47,7 +47,6 @@ __device__ __forceinline__ void transposed_reduce(float* x, int j) {
 // per SM it ran at 84 % of the measured copy bandwidth, with two and three at 99 %).
 // Group tiles of more than 4 query heads need the registers of a third CTA for their q and o
 // rows: they run two CTAs to an SM and take a third stage instead.
-constexpr int DEC_MAX_STAGES = 3;
 __host__ __device__ constexpr int dec_stages(int group_tile) { return group_tile > 4 ? 3 : 2; }
 __host__ __device__ constexpr int dec_ctas_per_sm(int group_tile) { return group_tile > 4 ? 2 : 3; }
 
