@@ -210,7 +210,10 @@ efim_status efim_append_prefill_step(const efim_cache_desc* cache, const efim_ba
  *   lse = log sum_c exp(lse_c),  o = sum_c exp(lse_c - lse) o_c.
  * max_ctx_len is an upper bound on every ctx_len[s] (<= 0: max_pages_per_seq *
  * page_size); it fixes the chunking, so no host copy of the lengths is needed.
- * ctx_len[s] == 0 gives out = 0, lse = -inf.  A device length beyond what the launch was
+ * ctx_len[s] == 0 gives out = 0, lse = -inf.  Query-head groups of up to 7 per kv head read
+ * the K/V pages once; larger groups are cut into tiles of 4 or 3 heads that each read them.
+ * (The kernel works on fp32 FMAs; from about 5 heads per kv head on a batch of decode rows is
+ * served faster by efim_append_prefill_attn as rows with new_len = 1, which is legal there.)  A device length beyond what the launch was
  * planned for (the chunks cover max_ctx_len rounded up to whole chunks, at most the block
  * table's capacity) is clamped to that and sets EFIM_DEV_BAD_POSITION; nothing outside the
  * workspace or the table is touched.

@@ -88,6 +88,18 @@ def test_bad_arguments_are_rejected_on_the_host():
     assert lib.efim_prefill_workspace_bytes(ctypes.byref(ok), ctypes.byref(bd)) > 0
     assert lib.efim_append_prefill_attn(ctypes.byref(ok), ctypes.byref(bd), 0x1000, 0x1000, None, 0.0,
                                         None, 0, None, None) == 4
+    # the one-call turn: k and v come together or not at all; the self-test refuses long limits
+    assert lib.efim_append_prefill_step(ctypes.byref(ok), ctypes.byref(bd), None, 0x1000, 0x1000, None, 0x1000, None,
+                                        0.0, None, 0, 0, None, 0, None, None) == 1
+    assert lib.efim_selftest_bounded_wait(10**9, 0x1000, None, None) == 1
+    assert lib.efim_selftest_bounded_wait(1000, None, None, None) == 1
+    # fragment spans: sizing call and argument checks
+    lib.efim_fim_fragment_spans.restype = ctypes.c_int64
+    lib.efim_fim_fragment_spans.argtypes = [ctypes.c_uint64, ctypes.c_int64, ctypes.c_int32, ctypes.c_int32,
+                                            ctypes.c_void_p, ctypes.c_int64]
+    assert lib.efim_fim_fragment_spans(1, 1000, 1, 200, None, 0) >= 6
+    assert lib.efim_fim_fragment_spans(1, 1000, 0, 200, None, 0) == -1
+    assert lib.efim_fim_fragment_spans(1, 10, 1, 200, None, 3) == -1
     # empty batch is a no-op
     bd0 = B._BatchDesc(0, 4, 0, None, None, None, None, None, None)
     assert lib.efim_kv_append(ctypes.byref(ok), ctypes.byref(bd0), None, None, None, None, None, None) == 0
