@@ -328,6 +328,35 @@ def test_garbage_beyond_the_context_and_odd_cached_values():
     H.assert_lse_close(lse_d.cpu().numpy(), lse, "decode beside NaN slots")
 
 
+def test_planned_prefill_with_resident_lists_can_be_captured_in_a_graph():
+    """With lists_resident = 1 the planned call copies nothing and only launches, so it can be
+    recorded into a CUDA graph (a model's per-layer loop); the replay gives the same bits."""
+    efim, H, _custom, _check_turn = _mods()
+    w = make_workload("cfg3", small=True)
+    dw = H.DeviceWorkload(w)
+    dw.gpu_kv_append()
+    plan = efim.efim_prefill_plan(dw.cache, dw.batch)
+    ws = torch.empty(max(efim.efim_prefill_workspace_bytes(dw.cache, dw.batch), 256), dtype=torch.uint8, device="cuda")
+    efim.efim_append_prefill_attn(dw.cache, dw.batch, dw.q, dw.out, dw.lse, 0.0, ws, dw.status, plan=plan)   # uploads the lists
+    torch.cuda.synchronize()
+    want_out, want_lse = dw.out.clone(), dw.lse.clone()
+    side = torch.cuda.Stream()
+    side.wait_stream(torch.cuda.current_stream())
+    graph = torch.cuda.CUDAGraph()
+    with torch.cuda.stream(side):
+        with torch.cuda.graph(graph, stream=side):
+            efim.efim_append_prefill_attn(dw.cache, dw.batch, dw.q, dw.out, dw.lse, 0.0, ws, dw.status, plan=plan,
+                                          lists_resident=True, stream=side)
+    torch.cuda.current_stream().wait_stream(side)
+    for _ in range(2):
+        dw.out.zero_()
+        dw.lse.zero_()
+        graph.replay()
+        torch.cuda.synchronize()
+        assert int(dw.status.item()) == 0
+        assert torch.equal(dw.out.view(torch.int16), want_out.view(torch.int16)) and torch.equal(dw.lse, want_lse)
+
+
 def test_bounded_wait_expires_and_reports():
     """One warp waits on a barrier nothing completes, with nothing in flight: after the
     limit the kernel sets EFIM_DEV_TIMEOUT and ends normally; the context stays usable."""
