@@ -6,7 +6,8 @@
 // (sequence, kv head) as two 128-row tiles, and streams the visible K/V range in
 // tiles of 128 keys (8 pages):
 //   warps 8,11 TMA producers (K tiles / V tiles): walk the block table, one tiled bulk-tensor
-//             copy per (page, 64-dim half) into a 5- or 6-entry shared-memory ring (128B swizzle)
+//             copy per page (16 slots x all dims of the kv head) into a 5- or 6-entry
+//             shared-memory ring (128B swizzle)
 //   warp 10   issues the tcgen05.mma for S_t = Q_t K^T into TMEM
 //   warp 9    issues the tcgen05.mma for O_t += P_t V (P read from TMEM)
 //   warps 0-7 two softmax groups, one per query tile, one TMEM lane (row) per thread:
@@ -54,12 +55,13 @@ __device__ __forceinline__ void umma_bf16_ts(uint32_t d_tmem, uint32_t a_tmem, u
       "r"(a_tmem), "l"(bdesc), "r"(idesc), "r"(accumulate)
       : "memory");
 }
-__device__ __forceinline__ void tma_load_4d(uint32_t dst, const CUtensorMap* map, uint32_t bar, int c0, int c1,
-                                            int c2, int c3) {
+// One (page, kv head) of a pool: coordinates (dim % 64, slot % 8, dim / 64, slot / 8, page * Hkv + head);
+// the first four are always 0 here (the box covers them whole).
+__device__ __forceinline__ void tma_load_page(uint32_t dst, const CUtensorMap* map, uint32_t bar, int page_head) {
   asm volatile(
-      "cp.async.bulk.tensor.4d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4, %5, %6}], [%2];" ::
-          "r"(dst),
-      "l"(map), "r"(bar), "r"(c0), "r"(c1), "r"(c2), "r"(c3)
+      "cp.async.bulk.tensor.5d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %3, %3, %3, %4}], "
+      "[%2];" ::"r"(dst),
+      "l"(map), "r"(bar), "r"(0), "r"(page_head)
       : "memory");
 }
 
@@ -126,15 +128,18 @@ __host__ __device__ constexpr uint32_t instr_desc(int n, int b_mn_major) {
          (static_cast<uint32_t>(n >> 3) << 17) | (static_cast<uint32_t>(BM >> 4) << 24);
 }
 
-// Shared-memory plan.  Operand tiles are [64-element half][128 rows][128 bytes],
-// 16-byte chunk c of row r stored at chunk position c ^ (r & 7) (the 128B swizzle
-// the tensor-map copies and the MMA descriptors both use).
+// Shared-memory plan.  A query tile is [64-element half][128 rows][128 bytes]; a K or V tile
+// is [8-key group][64-element half][8 keys][128 bytes], which is what one copy per page
+// writes (a page is two key groups).  In both, 16-byte chunk c of row r is stored at chunk
+// position c ^ (r & 7) (the 128B swizzle the tensor-map copies and the MMA descriptors use).
 template <int D>
 struct Smem {
   static constexpr int HALVES = D / 64;
   static constexpr int HALF_BYTES = 128 * 128;                  // 16 KB
   static constexpr int Q_BYTES = HALVES * HALF_BYTES;
   static constexpr int KV_BYTES = HALVES * HALF_BYTES;
+  static constexpr int GROUP_BYTES = HALVES * 1024;             // 8 keys of a K/V tile, all dims
+  static constexpr int PAGE_BYTES = 2 * GROUP_BYTES;            // one page = one copy
   static constexpr int Q_OFF = 0;
   static constexpr int KV_OFF = Q_OFF + NQ * Q_BYTES;
   static constexpr int BAR_OFF = KV_OFF + NSTAGE * KV_BYTES;
@@ -463,11 +468,11 @@ __device__ __forceinline__ void prefill_tc_body(const Params& p, const CUtensorM
   } else if (warp == 8 || warp == 11) {
     // ============================================================ TMA producers
     // Every bulk-tensor copy costs its issuing warp ~65 cycles and a 128-key tile takes
-    // 16 of them (one 2 KB box per page and 64-dim half), so one warp tops out near
-    // 30 GB/s.  Warp 8 therefore loads the K tiles and warp 11 the V tiles.
+    // 8 of them (one box per page: 16 slots x all dims of one kv head).  Warp 8 loads the
+    // K tiles and warp 11 the V tiles.
     const int my_which = warp == 8 ? 0 : 1;
     const int32_t* bt = p.block_table + (size_t)it.seq * p.max_pages_per_seq;
-    const int page_l = lane / HALVES, half_l = lane % HALVES;
+    const int page_l = lane;
     const CUtensorMap* my_map = my_which == 0 ? &map_k : &map_v;
     // does this lane fetch a page of tile jj (lanes beyond the tile's visible pages do not)?
     auto wanted = [&](int jj) {
@@ -476,7 +481,7 @@ __device__ __forceinline__ void prefill_tc_body(const Params& p, const CUtensorM
       const int keys = min(BN, kv_cap - tile * BN);
       const int npages = keys > 0 ? (keys + 15) >> 4 : 0;
       // (the last test only matters for a plan that does not belong to this block table)
-      return page_l < npages && lane < 8 * HALVES && tile * 8 + page_l < p.max_pages_per_seq;
+      return page_l < npages && tile * 8 + page_l < p.max_pages_per_seq;
     };
     auto lookup = [&](int jj, bool want) { return want ? __ldg(bt + (it.tile_begin + jj) * 8 + page_l) : -1; };
     // the block-table read is a dependent global load in front of every copy: fetch it two tiles ahead
@@ -494,24 +499,24 @@ __device__ __forceinline__ void prefill_tc_body(const Params& p, const CUtensorM
       const bool bad = want && !ok;                          // an id outside the pool: reported, never dereferenced
       const uint32_t okmask = __ballot_sync(0xffffffffu, ok);
       const bool any_bad = __any_sync(0xffffffffu, bad);
-      const uint32_t bytes = __popc(okmask) * 2048u;
+      const uint32_t bytes = __popc(okmask) * (uint32_t)L::PAGE_BYTES;
       const int slot = ld % nst, use = ld / nst;
       mbar_wait(bar(BAR_EMPTY + slot), (use & 1) ^ 1, abort_flag, p.status, p.wait_ns);
-      const uint32_t dst_off = ring_off + slot * L::KV_BYTES + half_l * L::HALF_BYTES + page_l * 2048;
+      const uint32_t dst_off = ring_off + slot * L::KV_BYTES + page_l * L::PAGE_BYTES;
       if (any_bad) {
         // the page's 16 keys are replaced by zeros (score 0, value 0), so the tile holds nothing
         // undefined; written with ordinary stores, made visible to the tensor core's reads
         if (bad) {
           if (my_which == 0 && p.status) atomicOr(p.status, EFIM_DEV_BAD_PAGE);
           uint4* z = reinterpret_cast<uint4*>(smem_gen + dst_off);
-          for (int i = 0; i < 128; ++i) z[i] = make_uint4(0, 0, 0, 0);
+          for (int i = 0; i < L::PAGE_BYTES / 16; ++i) z[i] = make_uint4(0, 0, 0, 0);
           fence_async_smem();
         }
         __syncwarp();
       }
       if (lane == 0) mbar_expect_tx(bar(BAR_FULL + slot), bytes);
       __syncwarp();
-      if (ok) tma_load_4d(smem_base + dst_off, my_map, bar(BAR_FULL + slot), half_l * 64, 0, it.kvh, pid);
+      if (ok) tma_load_page(smem_base + dst_off, my_map, bar(BAR_FULL + slot), pid * p.Hkv + it.kvh);
     }
     // if the CTA gave up, let copies that are still in flight land before shared memory goes away
     if (*abort_flag) {
@@ -535,19 +540,22 @@ __device__ __forceinline__ void prefill_tc_body(const Params& p, const CUtensorM
     mbar_wait(bar(BAR_Q + 0), 0, abort_flag, p.status, p.wait_ns);
     if (dual) mbar_wait(bar(BAR_Q + 1), 0, abort_flag, p.status, p.wait_ns);
     tc_fence_after();
-    // Descriptors: the high word is fixed (SBO 1024, version 1, 128B swizzle); the low
-    // word is (address >> 4) | LBO << 16, so stepping through a tile is one add.
-    constexpr uint32_t DESC_HI = (1024u >> 4) | (1u << 14) | (2u << 29);
+    // Descriptors: the high word is fixed (SBO = distance between 8-row groups: 1024 in a
+    // query tile, GROUP_BYTES in a K/V tile; version 1; 128B swizzle); the low word is
+    // (address >> 4) | LBO << 16, so stepping through a tile is one add.
+    constexpr uint32_t DESC_HI_Q = (1024u >> 4) | (1u << 14) | (2u << 29);
+    constexpr uint32_t DESC_HI_KV = ((uint32_t)L::GROUP_BYTES >> 4) | (1u << 14) | (2u << 29);
     constexpr uint32_t LBO_K = 1u << 16;                                           // K-major: LBO unused
-    constexpr uint32_t LBO_V = (uint32_t)(L::HALF_BYTES >> 4) << 16;              // MN-major: next 64 dims
-    auto desc = [&](uint32_t lo) { return (static_cast<uint64_t>(DESC_HI) << 32) | lo; };
+    constexpr uint32_t LBO_V = (1024u >> 4) << 16;                                 // MN-major: next 64 dims
+    auto desc_q = [&](uint32_t lo) { return (static_cast<uint64_t>(DESC_HI_Q) << 32) | lo; };
+    auto desc = [&](uint32_t lo) { return (static_cast<uint64_t>(DESC_HI_KV) << 32) | lo; };
     const uint32_t kv_lo = kv_base >> 4, q_lo = (q_base >> 4) | LBO_K;
     // O_st (+)= P_st V for half h (keys 64h..64h+63) of KV tile n (ring load 2n+1); P from TMEM
     auto issue_pv_half = [&](int st, int n, int h, uint32_t first) {
       const uint32_t v_lo = (kv_lo + (ld_v(n) % nst) * (L::KV_BYTES >> 4)) | LBO_V;
 #pragma unroll
       for (int k = 4 * h; k < 4 * h + 4; ++k)
-        umma_bf16_ts(tmem_O + st * D, tmem_S + st * BN + k * 8, desc(v_lo + k * (2048 >> 4)), IDESC_PV,
+        umma_bf16_ts(tmem_O + st * D, tmem_S + st * BN + k * 8, desc(v_lo + k * (2 * L::GROUP_BYTES >> 4)), IDESC_PV,
                      (!first || k > 0) ? 1u : 0u);
     };
     auto issue_qk = [&](int st, int n) {
@@ -555,8 +563,9 @@ __device__ __forceinline__ void prefill_tc_body(const Params& p, const CUtensorM
       const uint32_t a_lo = q_lo + (dual ? st : 0) * (L::Q_BYTES >> 4);
 #pragma unroll
       for (int k = 0; k < D / 16; ++k) {
-        const uint32_t off = ((k >> 2) * L::HALF_BYTES + (k & 3) * 32) >> 4;
-        umma_bf16(tmem_S + st * BN, desc(a_lo + off), desc(k_lo + off), IDESC_QK, k > 0 ? 1u : 0u);
+        const uint32_t off_q = ((k >> 2) * L::HALF_BYTES + (k & 3) * 32) >> 4;
+        const uint32_t off_k = ((k >> 2) * 1024 + (k & 3) * 32) >> 4;
+        umma_bf16(tmem_S + st * BN, desc_q(a_lo + off_q), desc(k_lo + off_k), IDESC_QK, k > 0 ? 1u : 0u);
       }
     };
     // V rows past the visible range hold stale or foreign data; P is 0 there but
@@ -569,7 +578,8 @@ __device__ __forceinline__ void prefill_tc_body(const Params& p, const CUtensorM
         const int chunks = (BN - first) * 8 * HALVES;       // 16-byte chunks to clear
         for (int idx = lane; idx < chunks; idx += 32) {
           const int h = idx / ((BN - first) * 8), rem = idx % ((BN - first) * 8);
-          *reinterpret_cast<uint4*>(vb + h * L::HALF_BYTES + (first + (rem >> 3)) * 128 + ((rem & 7) << 4)) =
+          const int key = first + (rem >> 3);
+          *reinterpret_cast<uint4*>(vb + (key >> 3) * L::GROUP_BYTES + h * 1024 + (key & 7) * 128 + ((rem & 7) << 4)) =
               make_uint4(0, 0, 0, 0);
         }
         fence_async_smem();
@@ -846,16 +856,18 @@ static EncodeTiledFn encode_fn() {
   return fn;
 }
 
-// Pool [pages][Hkv][16][D] bf16 as a 4-D tensor (d, slot, head, page); one box =
-// 64 dims x 16 slots of one (page, head) = 2 KB, 128-byte swizzled.
+// Pool [pages][Hkv][16][D] bf16 as a 5-D tensor (dim % 64, slot % 8, dim / 64, slot / 8,
+// page * Hkv + head); one box = the 16 slots x D dims of one (page, head), written to shared
+// memory as [slot / 8][dim / 64][slot % 8][64 dims], 128-byte swizzled.
 static bool make_pool_map(CUtensorMap* m, void* pool, int pages, int Hkv, int D) {
   EncodeTiledFn fn = encode_fn();
   if (!fn) return false;
-  const cuuint64_t dims[4] = {(cuuint64_t)D, 16, (cuuint64_t)Hkv, (cuuint64_t)pages};
-  const cuuint64_t strides[3] = {(cuuint64_t)D * 2, (cuuint64_t)D * 2 * 16, (cuuint64_t)D * 2 * 16 * Hkv};
-  const cuuint32_t box[4] = {64, 16, 1, 1};
-  const cuuint32_t estr[4] = {1, 1, 1, 1};
-  return fn(m, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 4, pool, dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
+  const cuuint64_t row = (cuuint64_t)D * 2;
+  const cuuint64_t dims[5] = {64, 8, (cuuint64_t)D / 64, 2, (cuuint64_t)pages * Hkv};
+  const cuuint64_t strides[4] = {row, 128, 8 * row, 16 * row};
+  const cuuint32_t box[5] = {64, 8, (cuuint32_t)D / 64, 2, 1};
+  const cuuint32_t estr[5] = {1, 1, 1, 1, 1};
+  return fn(m, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 5, pool, dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
             CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
             CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }

@@ -13,9 +13,11 @@ constexpr int NSTAGE = 5;      // K/V ring entries (one K or V tile of 128 keys 
 constexpr int NSTAGE_MAX = 6;  // ring entries when there is a single query tile (the other tile's space is used)
 constexpr int THREADS = 384;   // 2 softmax warpgroups + 1 service warpgroup (2 TMA warps, 2 MMA warps)
 // Register split (setmaxnreg): the block launches with 168 registers per thread
-// (65536 / 384, rounded to 8) = 64512 in total; 2 x 128 x 216 + 128 x 64 = 63488 fits.
+// (65536 / 384, rounded to 8) = 64512 in total; 2 x 128 x 216 + 128 x 72 = 64512 uses them all
+// (the sum must not exceed the launch total: an increase beyond it would wait forever).  With
+// 64 registers the service warps spilled a few words inside the MMA-issuing loop.
 constexpr int REGS_SOFTMAX = 216;
-constexpr int REGS_SERVICE = 64;
+constexpr int REGS_SERVICE = 72;
 
 // One CTA's work: packed rows [row0, row0 + 256) of (seq, kv head) against KV tiles
 // [tile_begin, tile_end).  Packed row R = token * G + head-in-group.  The sequence's
