@@ -58,7 +58,8 @@ extern "C" {
 typedef enum {
   EFIM_OK = 0,
   EFIM_ERR_INVALID_ARG = 1,   /* null pointer, negative size, H_q % H_kv != 0, bad alignment */
-  EFIM_ERR_UNSUPPORTED = 2,   /* head_dim / page_size outside the supported set            */
+  EFIM_ERR_UNSUPPORTED = 2,   /* head_dim / page_size outside the supported set; more than 32767 kv heads
+                                 or num_pages * num_kv_heads above 2^31 - 1                  */
   EFIM_ERR_OUT_OF_RANGE = 3,  /* a host-visible length exceeds max_pages_per_seq*page_size  */
   EFIM_ERR_WORKSPACE = 4,     /* workspace_bytes smaller than the *_workspace_bytes() answer */
   EFIM_ERR_CUDA = 5,          /* a CUDA runtime/driver call failed (launch, copy, tensor map) */

@@ -28,6 +28,8 @@ inline efim_status check_cache(const efim_cache_desc* c) {
   if (c->num_pages <= 0 || c->num_q_heads <= 0 || c->num_kv_heads <= 0) return EFIM_ERR_INVALID_ARG;
   if (c->num_q_heads % c->num_kv_heads != 0) return EFIM_ERR_INVALID_ARG;
   if (c->num_kv_heads > 32767) return EFIM_ERR_UNSUPPORTED;
+  // a (page, kv head) pair is one 32-bit coordinate of the prefill kernel's page copies
+  if ((long long)c->num_pages * c->num_kv_heads > 0x7fffffffLL) return EFIM_ERR_UNSUPPORTED;
   if (c->page_size != 16) return EFIM_ERR_UNSUPPORTED;
   if (c->head_dim != 64 && c->head_dim != 128) return EFIM_ERR_UNSUPPORTED;
   if ((reinterpret_cast<uintptr_t>(c->d_k_pool) & 127) || (reinterpret_cast<uintptr_t>(c->d_v_pool) & 127))

@@ -64,6 +64,10 @@ def test_bad_arguments_are_rejected_on_the_host():
         st = lib.efim_decode_attn(ctypes.byref(bad), 1, 0x1000, 16, 0x1000, 4, 0x1000, 0x1000, None, 0.0,
                                   None, 0, None, None)
         assert st == code
+    # a (page, kv head) pair has to fit one 32-bit coordinate
+    big = B._CacheDesc(0x10000, 0x20000, 1 << 28, 16, 8, 8, 128)
+    assert lib.efim_decode_attn(ctypes.byref(big), 1, 0x1000, 16, 0x1000, 4, 0x1000, 0x1000, None, 0.0,
+                                None, 0, None, None) == 2
     # null inputs
     assert lib.efim_decode_attn(ctypes.byref(ok), 1, None, 16, 0x1000, 4, 0x1000, 0x1000, None, 0.0,
                                 None, 0, None, None) == 1
