@@ -704,7 +704,7 @@ namespace {
 // bytes; every CTA pays for its set-up, query load, pipeline fill and epilogue; a split
 // adds the partials' round trip and the merge launch.
 constexpr long long COST_TILE_DUAL = 21, COST_TILE_SINGLE = 15, COST_CTA = 100, COST_PARTIAL = 8, COST_MERGE = 80;
-constexpr long long COST_TILE_SINGLE_TAIL = 12;    // a one-tile CTA's tile when the GPU is no longer full
+constexpr long long COST_TILE_SINGLE_TAIL = 9;     // a one-tile CTA's tile when the GPU is no longer full
 
 // Finish time of the launch if the K/V range of every sequence is cut into chunks of
 // `chunk_tiles` tiles: the hardware hands CTAs, longest first, to whichever SM is free.
@@ -818,9 +818,10 @@ Plan make_plan(const efim_cache_desc* c, const efim_batch_desc* b, WorkItem* ite
     } else {
       // Few waves: costliest first, so the tail of the launch is made of cheap items.  A tile
       // costs a two-tile CTA (bound by its softmax) 2.1 us wherever it runs; a one-tile CTA is
-      // bound by its K/V bytes and speeds up once SMs fall idle at the end of the launch, so
-      // it is weighted 1.2 us here, not the 1.5 us of a full GPU (cfg2: 0.305 ms ordered by
-      // tile count, 0.290 by cost at 2.1 : 1.5, 0.281 at 2.1 : 1.2).
+      // bound by its K/V bytes and speeds up once SMs fall idle at the end of the launch (measured:
+      // 0.89 us per tile with 8 to 32 such CTAs on the GPU, 1.5 us with 148), so it is weighted
+      // 0.9 us here (cfg2: 0.305 ms ordered by tile count, 0.290 by cost at 2.1 : 1.5, 0.281 at
+      // 2.1 : 1.2; 2.1 : 0.9 is 3-5 % faster still on three of four other draws of cfg2).
       auto cost = [G](const WorkItem& w) {
         const long long rows_here = std::min<long long>((long long)w.new_len * G - w.row0, NQ * BM);
         return (long long)(w.tile_end - w.tile_begin) * (rows_here > BM ? COST_TILE_DUAL : COST_TILE_SINGLE_TAIL);
