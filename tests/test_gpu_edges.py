@@ -114,12 +114,15 @@ def test_kv_append_reports_bad_page_and_bad_position_and_skips_them():
     assert not torch.equal(dw2.k_pool[pg4].view(torch.int16), before[pg4].view(torch.int16))
 
 
+@pytest.mark.parametrize("head_dim", [128, 64])
 @pytest.mark.parametrize("bad_id", ["beyond_pool", "negative"])
-def test_prefill_reports_bad_page_keeps_other_rows(bad_id):
+def test_prefill_reports_bad_page_keeps_other_rows(bad_id, head_dim):
     """A block-table entry outside the pool among the pages a row sees: EFIM_DEV_BAD_PAGE,
-    finite output everywhere, and the sequences that do not see the entry are unaffected."""
+    finite output everywhere, the sequences that do not see the entry are unaffected, and the
+    sequence that does gets what the header promises: the page's 16 keys count as zero keys
+    with zero values."""
     efim, H, _custom, _check_turn = _mods()
-    w = _custom(8, 2, 128, [300, 200, 500], [140, 60, 9])
+    w = _custom(8, 2, head_dim, [300, 200, 500], [140, 60, 9])
     dw = H.DeviceWorkload(w)
     dw.gpu_kv_append()
     table = dw.batch.d_block_table.clone()
@@ -133,6 +136,13 @@ def test_prefill_reports_bad_page_keeps_other_rows(bad_id):
     ref = dw.oracle_turn([0, 2])
     H.assert_attn_close(H.torch_to_bits(dw.out)[ref["rows"]], ref["o"], "rows that do not see the bad entry")
     H.assert_lse_close(dw.lse.cpu().numpy()[ref["rows"]], ref["lse"], "rows that do not see the bad entry")
+    one = dw.oracle_turn([1])
+    kp, vp = one["k_pool"].copy(), one["v_pool"].copy()
+    kp[one["bt"][0, 6]] = 0                                   # bf16 bit pattern 0 = +0.0
+    vp[one["bt"][0, 6]] = 0
+    o, lse = orc.append_prefill_attention(one["q_rot"], kp, vp, one["bt"], one["cached"], one["new"], w.num_q_heads)
+    H.assert_attn_close(H.torch_to_bits(dw.out)[one["rows"]], o, "rows that see the bad entry as zero keys")
+    H.assert_lse_close(dw.lse.cpu().numpy()[one["rows"]], lse, "rows that see the bad entry as zero keys")
 
 
 @pytest.mark.parametrize("static", [False, True])
