@@ -175,3 +175,49 @@ def test_prefill_plan_blob_sizes_and_errors():
     none = _batch_desc([100, 200], [0, 0], 32)
     assert lib.efim_prefill_plan_bytes(ctypes.byref(cache), ctypes.byref(none)) == 256
     assert lib.efim_prefill_plan(ctypes.byref(cache), ctypes.byref(none), buf.ctypes.data, 256) == 0
+
+
+_ITEM = np.dtype([("seq", "i4"), ("kvh", "i2"), ("chunk", "i2"), ("row0", "i4"), ("tile_begin", "i4"),
+                  ("tile_end", "i4"), ("cached", "i4"), ("new_len", "i4"), ("tok0", "i4")])
+
+
+def _plan_items(lib, cache, batch):
+    lib.efim_prefill_plan_bytes.restype = ctypes.c_size_t
+    n = lib.efim_prefill_plan_bytes(ctypes.byref(cache), ctypes.byref(batch))
+    buf = np.zeros(n, np.uint8)
+    assert lib.efim_prefill_plan(ctypes.byref(cache), ctypes.byref(batch), buf.ctypes.data, n) == 0
+    n_items = int(np.frombuffer(buf[:64].tobytes(), np.int32)[6])
+    return np.frombuffer(buf[256:256 + 32 * n_items].tobytes(), _ITEM)
+
+
+def test_prefill_work_list_covers_every_row_and_key_once_and_is_ordered_by_cost():
+    """The work list of a ragged batch (a few waves of CTAs): every (sequence, kv head, block
+    of 256 packed rows) appears with the whole key range its last row sees, cut into
+    disjoint chunks if at all; items carry their sequence's lengths and first query row; and
+    the launch order is costliest first, a tile of a two-tile item (more than 128 rows)
+    weighing 2.1 and a tile of a one-tile item 0.9."""
+    lib = efim.load_library()
+    Hq, Hkv = 8, 2
+    G = Hq // Hkv
+    cache = _cache_desc(Hq=Hq, Hkv=Hkv)
+    cached = [3000, 500, 7000, 40, 2222, 900, 5000, 64]
+    new = [200, 17, 40, 130, 1, 64, 33, 90]
+    items = _plan_items(lib, cache, _batch_desc(cached, new, 512))
+    tok0 = np.concatenate([[0], np.cumsum(new)])
+    seen = {}
+    for it in items:
+        s = int(it["seq"])
+        assert (it["cached"], it["new_len"], it["tok0"]) == (cached[s], new[s], tok0[s])
+        assert 0 <= it["kvh"] < Hkv and it["row0"] % 256 == 0 and it["row0"] < new[s] * G
+        seen.setdefault((s, int(it["kvh"]), int(it["row0"])), []).append((int(it["tile_begin"]), int(it["tile_end"])))
+    want = {(s, h, r0) for s in range(len(new)) for h in range(Hkv) for r0 in range(0, new[s] * G, 256)}
+    assert set(seen) == want
+    for (s, h, r0), ranges in seen.items():
+        last_tok = (min(new[s] * G, r0 + 256) - 1) // G
+        tiles = -(-(cached[s] + last_tok + 1) // 128)
+        ranges.sort()
+        assert ranges[0][0] == 0 and ranges[-1][1] == tiles
+        assert all(a[1] == b[0] for a, b in zip(ranges, ranges[1:]))      # disjoint, no gap
+    rows_here = np.minimum(items["new_len"] * G - items["row0"], 256)
+    cost = (items["tile_end"] - items["tile_begin"]) * np.where(rows_here > 128, 21, 9)
+    assert (np.diff(cost) <= 0).all()
