@@ -155,12 +155,135 @@ enum {
   BAR_COUNT = 12 + 2 * NSTAGE_MAX
 };
 
+// Epilogue of the 32-row shape: the eight (max, sum, O) states of query row `lane`, left in
+// shared memory as [state][row][XROW], are merged; this thread finishes D/8 dims of the row
+// (slice `sidx`) and stores them (final output, or a chunk's partial).  Out of line: it runs
+// once per CTA and its registers should not count against the loops of the caller.
+template <int D>
+__device__ __noinline__ void tiny_merge_store(uint16_t* out, float* lse, float* part_o, float* part_lse, int s_max,
+                                              const float* xb, int lane, int sidx, bool valid, int chunk,
+                                              size_t row_off, size_t th) {
+  using L = Smem<D>;
+  constexpr int DS = D / 8;
+  float M = -INFINITY;
+#pragma unroll
+  for (int q = 0; q < 8; ++q) M = fmaxf(M, xb[(size_t)(q * 32 + lane) * L::XROW + D]);
+  float Lt = 0.f, acc[DS];
+#pragma unroll
+  for (int d = 0; d < DS; ++d) acc[d] = 0.f;
+#pragma unroll
+  for (int q = 0; q < 8; ++q) {
+    const float* row = xb + (size_t)(q * 32 + lane) * L::XROW;
+    const float lq = row[D + 1];
+    const float wq = lq > 0.f ? ex2(row[D] - M) : 0.f;
+    Lt = fmaf(lq, wq, Lt);
+#pragma unroll
+    for (int d = 0; d < DS; d += 4) {
+      const float4 x = *reinterpret_cast<const float4*>(row + sidx * DS + d);
+      acc[d] = fmaf(x.x, wq, acc[d]);
+      acc[d + 1] = fmaf(x.y, wq, acc[d + 1]);
+      acc[d + 2] = fmaf(x.z, wq, acc[d + 2]);
+      acc[d + 3] = fmaf(x.w, wq, acc[d + 3]);
+    }
+  }
+  const float inv = Lt > 0.f ? 1.f / Lt : 0.f;
+  const float lse2 = Lt > 0.f ? M + log2f(Lt) : -INFINITY;
+  if (!valid) return;
+  if (chunk < 0) {
+    uint4* dst = reinterpret_cast<uint4*>(out + row_off + sidx * DS);
+#pragma unroll
+    for (int d = 0; d < DS; d += 8)
+      dst[d / 8] = make_uint4(pack_bf16x2(acc[d] * inv, acc[d + 1] * inv), pack_bf16x2(acc[d + 2] * inv, acc[d + 3] * inv),
+                              pack_bf16x2(acc[d + 4] * inv, acc[d + 5] * inv), pack_bf16x2(acc[d + 6] * inv, acc[d + 7] * inv));
+    if (sidx == 0 && lse) lse[th] = lse2 * 0.6931471805599453f;
+  } else {
+    float4* dst = reinterpret_cast<float4*>(part_o + (th * s_max + chunk) * D + sidx * DS);
+#pragma unroll
+    for (int d = 0; d < DS; d += 4)
+      dst[d / 4] = make_float4(acc[d] * inv, acc[d + 1] * inv, acc[d + 2] * inv, acc[d + 3] * inv);
+    if (sidx == 0) part_lse[th * s_max + chunk] = lse2;
+  }
+}
+
+// O row of every lane of the warp *= alpha (the rare rescale of the 32-row shape; kept out
+// of line so that its 32 registers do not count against the loop that calls it).
+template <int D>
+__device__ __noinline__ void rescale_o_row(uint32_t o_addr, float alpha) {
+#pragma unroll
+  for (int c0 = 0; c0 < D; c0 += 32) {
+    uint32_t o[32];
+    EFIM_TMEM_LD32(o_addr + c0, o);
+    tmem_wait_ld();
+#pragma unroll
+    for (int c = 0; c < 32; ++c) o[c] = __float_as_uint(__uint_as_float(o[c]) * alpha);
+    EFIM_TMEM_ST32(o_addr + c0, o);
+  }
+}
+
+// One query row -> its row of a shared-memory query tile (swizzled), zero for a row past the
+// sequence; with a rotary table the row is rotated by its position on the way (the
+// arithmetic of efim_kv_append).  `qrow` = tile base + 128 * tile row, `r` = tile row.
+template <int D>
+__device__ __forceinline__ void q_row_to_smem(const Params& p, uint8_t* qrow, int r, bool valid, int pos,
+                                              size_t row_off) {
+  using L = Smem<D>;
+  const uint4* src = reinterpret_cast<const uint4*>(p.q + row_off);
+  auto put = [&](int c, uint4 v) {
+    *reinterpret_cast<uint4*>(qrow + (c >> 3) * L::HALF_BYTES + (((c & 7) ^ (r & 7)) << 4)) = v;
+  };
+  if (p.cos_sin == nullptr || !valid) {
+#pragma unroll
+    for (int c = 0; c < D / 8; ++c) {
+      uint4 v = make_uint4(0, 0, 0, 0);
+      if (valid) v = __ldg(src + c);
+      put(c, v);
+    }
+  } else if (pos >= p.max_position) {
+    if (p.status) atomicOr(p.status, EFIM_DEV_BAD_POSITION);
+#pragma unroll
+    for (int c = 0; c < D / 8; ++c) put(c, make_uint4(0, 0, 0, 0));
+  } else {
+    const float* cs = p.cos_sin + (size_t)pos * D;
+    if (!p.interleaved) {
+#pragma unroll
+      for (int c = 0; c < D / 16; ++c) {
+        uint4 a = __ldg(src + c), b = __ldg(src + c + D / 16);
+        float cf[8], sf[8];
+        *reinterpret_cast<float4*>(cf) = __ldg(reinterpret_cast<const float4*>(cs + c * 8));
+        *reinterpret_cast<float4*>(cf + 4) = __ldg(reinterpret_cast<const float4*>(cs + c * 8 + 4));
+        *reinterpret_cast<float4*>(sf) = __ldg(reinterpret_cast<const float4*>(cs + D / 2 + c * 8));
+        *reinterpret_cast<float4*>(sf + 4) = __ldg(reinterpret_cast<const float4*>(cs + D / 2 + c * 8 + 4));
+        rotate8(a, b, cf, sf);
+        put(c, a);
+        put(c + D / 16, b);
+      }
+    } else {
+#pragma unroll
+      for (int c = 0; c < D / 8; ++c) {
+        uint4 a = __ldg(src + c);
+        float cf[4], sf[4];
+        *reinterpret_cast<float4*>(cf) = __ldg(reinterpret_cast<const float4*>(cs + c * 4));
+        *reinterpret_cast<float4*>(sf) = __ldg(reinterpret_cast<const float4*>(cs + D / 2 + c * 4));
+        rotate4_interleaved(a, cf, sf);
+        put(c, a);
+      }
+    }
+  }
+}
+
 // Two softmax groups ("streams") run per CTA.  With more than 128 rows, stream t
 // owns query tile t and both walk every KV tile.  With 128 rows or fewer there is
 // one query tile; stream 0 takes the even KV tiles and stream 1 the odd ones, each
 // with its own running (max, sum, O), and the two states are merged at the end -
 // the tensor core then still works on one stream while the other does its softmax.
-template <int D, bool DUAL>
+//
+// MODE 0: one query tile (33..128 rows); 1: two query tiles; 2: at most 32 rows (one-token rows of
+// a mixed batch, short `inc`s): the one query tile holds the rows four times, once per 32-lane
+// quarter, and the softmax warp of quarter w takes keys 32w..32w+31 of every tile with a
+// running (max, sum, O) of its own - a quarter of the exponentials per thread and tile, so the
+// two alternating streams turn a tile round in about half the time; the eight states of a row
+// (2 streams x 4 quarters) are merged at the end through shared memory.
+template <int D, int MODE>
 __device__ __forceinline__ void prefill_tc_body(const Params& p, const CUtensorMap& map_k, const CUtensorMap& map_v,
                                                 const WorkItem& it) {
   using L = Smem<D>;
@@ -178,7 +301,8 @@ __device__ __forceinline__ void prefill_tc_body(const Params& p, const CUtensorM
   const int C = it.cached, N = it.new_len, tok0 = it.tok0;
   const int rows_total = N * G;
   const int rows_here = min(NQ * BM, rows_total - it.row0);
-  constexpr bool dual = DUAL;                                // two query tiles (rows_here > BM)
+  constexpr bool dual = MODE == 1;                           // two query tiles (rows_here > BM)
+  constexpr bool tiny = MODE == 2;                           // at most 32 rows, held four times
   const int i_last = (it.row0 + rows_here - 1) / G;          // last token of this CTA
   const int kv_cap = C + i_last + 1;                         // keys any row here may see
   const int nt = it.tile_end - it.tile_begin;
@@ -231,7 +355,120 @@ __device__ __forceinline__ void prefill_tc_body(const Params& p, const CUtensorM
     asm volatile("setmaxnreg.inc.sync.aligned.u32 %0;" ::"n"(REGS_SOFTMAX));
   }
 
-  if (warp < 8) {
+  if (warp < 8 && tiny) {
+    // ============================================================ softmax groups, 32-row shape
+    const int st = warp >> 2, w = warp & 3;                 // stream, 32-lane quarter
+    const int my_cnt = st == 0 ? cnt0 : cnt1;
+    const int r = w * 32 + lane;                            // tile row == TMEM lane; the query row is `lane`
+    const int R = it.row0 + lane;
+    const bool valid = R < rows_total;
+    const int i_tok = valid ? R / G : 0;
+    const int g = valid ? R - i_tok * G : 0;
+    const int vis = valid ? C + i_tok + 1 : kv_cap;
+    const size_t row_off = ((size_t)(tok0 + i_tok) * p.Hq + (size_t)it.kvh * G + g) * D;
+    if (st == 0) {
+      q_row_to_smem<D>(p, smem_gen + L::Q_OFF + r * 128, r, valid, C + i_tok, row_off);
+      fence_async_smem();
+      mbar_arrive(bar(BAR_Q + 0));
+    }
+    const uint32_t lane_addr = (uint32_t)(w * 32) << 16;
+    const uint32_t s_addr = tmem_S + lane_addr + st * BN;
+    const uint32_t o_addr = tmem_O + lane_addr + st * D;
+    float m_ref = -INFINITY, l_sum = 0.f;
+    for (int k = 0; k < my_cnt; ++k) {
+      mbar_wait(bar(BAR_S + st), k & 1, abort_flag, p.status, p.wait_ns);
+      tc_fence_after();
+      uint32_t s[32];
+      EFIM_TMEM_LD32(s_addr + 32 * w, s);
+      tmem_wait_ld();
+      // P = bf16 pairs in columns 0..63 of this stream's S; this quarter's keys are columns
+      // 16w..16w+15 of it, the rest of the row is zero.  The 32-column half without values goes first.
+      uint32_t z[32];
+#pragma unroll
+      for (int c = 0; c < 32; ++c) z[c] = 0u;
+      EFIM_TMEM_ST32(s_addr + (w < 2 ? 32 : 0), z);
+      tmem_wait_st();
+      tc_fence_before();
+      mbar_arrive(bar(BAR_P + 2 * st + (w < 2 ? 1 : 0)));
+      const int kv0 = (it.tile_begin + 2 * k + st) * BN + 32 * w;
+      if (__any_sync(0xffffffffu, kv0 + 32 > vis)) {
+#pragma unroll
+        for (int c = 0; c < 32; ++c)
+          if (kv0 + c >= vis) s[c] = 0xff800000u;           // -inf
+      }
+      float mx4[4];
+#pragma unroll
+      for (int a = 0; a < 4; ++a) mx4[a] = __uint_as_float(s[a]);
+#pragma unroll
+      for (int c = 4; c < 32; c += 4)
+#pragma unroll
+        for (int a = 0; a < 4; ++a) mx4[a] = fmaxf(mx4[a], __uint_as_float(s[c + a]));
+      const float m_new = fmaxf(fmaxf(mx4[0], mx4[1]), fmaxf(mx4[2], mx4[3])) * p.scale_log2;
+      // lazy rescale, as in the other shapes (O is quiet: S(k) ready means PV(k-1) has landed)
+      const bool grow = m_new > m_ref + 8.f;
+      if (k == 0) {
+        m_ref = m_new;
+      } else if (__any_sync(0xffffffffu, grow)) {
+        const float alpha = grow ? ex2(m_ref - m_new) : 1.f;
+        if (grow) m_ref = m_new;
+        l_sum *= alpha;
+        rescale_o_row<D>(o_addr, alpha);
+      }
+      const float neg_m = (m_ref == -INFINITY) ? 0.f : -m_ref;
+      float ls[4] = {0.f, 0.f, 0.f, 0.f};
+      uint32_t v[16];
+#pragma unroll
+      for (int e = 0; e < 16; ++e) {
+        const float p0 = ex2(fmaf(__uint_as_float(s[2 * e]), p.scale_log2, neg_m));
+        const float p1 = ex2(fmaf(__uint_as_float(s[2 * e + 1]), p.scale_log2, neg_m));
+        ls[e & 3] += p0 + p1;
+        v[e] = pack_bf16x2(p0, p1);
+      }
+      uint32_t wv[32];
+      if (w & 1) {
+#pragma unroll
+        for (int e = 0; e < 16; ++e) { wv[e] = 0u; wv[16 + e] = v[e]; }
+      } else {
+#pragma unroll
+        for (int e = 0; e < 16; ++e) { wv[e] = v[e]; wv[16 + e] = 0u; }
+      }
+      EFIM_TMEM_ST32(s_addr + (w < 2 ? 0 : 32), wv);
+      tmem_wait_st();
+      tc_fence_before();
+      mbar_arrive(bar(BAR_P + 2 * st + (w < 2 ? 0 : 1)));
+      l_sum += (ls[0] + ls[1]) + (ls[2] + ls[3]);
+    }
+    // ---- epilogue: all MMAs of both streams done (the ring is quiet), then the eight states of
+    // every row meet in the ring's shared memory
+    mbar_wait(bar(BAR_O + 0), 0, abort_flag, p.status, p.wait_ns);
+    if (cnt1 > 0) mbar_wait(bar(BAR_O + 1), 0, abort_flag, p.status, p.wait_ns);
+    tc_fence_after();
+    static_assert(8 * 32 * L::XROW * 4 <= NSTAGE_MAX * L::KV_BYTES, "the eight states must fit in the ring");
+    float* xb = reinterpret_cast<float*>(smem_gen + ring_off);          // [8 states][32 rows][XROW]
+    const int sidx = st * 4 + w;
+    float* mine = xb + (size_t)(sidx * 32 + lane) * L::XROW;
+    const bool have = my_cnt > 0 && l_sum > 0.f;
+    if (lane < 32) {
+      mine[D] = have ? m_ref : -INFINITY;
+      mine[D + 1] = have ? l_sum : 0.f;
+    }
+#pragma unroll
+    for (int c0 = 0; c0 < D; c0 += 32) {
+      uint32_t o[32];
+      if (my_cnt > 0) {                                                 // warp-uniform: the load is warp-wide
+        EFIM_TMEM_LD32(o_addr + c0, o);
+        tmem_wait_ld();
+      }
+#pragma unroll
+      for (int c = 0; c < 32; c += 4)
+        *reinterpret_cast<uint4*>(mine + c0 + c) =
+            have ? make_uint4(o[c], o[c + 1], o[c + 2], o[c + 3]) : make_uint4(0, 0, 0, 0);
+    }
+    asm volatile("bar.sync 1, 256;" ::: "memory");
+    tiny_merge_store<D>(p.out, p.lse, p.part_o, p.part_lse, p.s_max, xb, lane, sidx, valid, it.chunk, row_off,
+                        (size_t)(tok0 + i_tok) * p.Hq + (size_t)it.kvh * G + g);
+    tc_fence_before();
+  } else if (warp < 8) {
     // ============================================================ softmax groups
     const int st = warp >> 2;                               // stream
     const int my_cnt = st == 0 ? cnt0 : cnt1;
@@ -575,13 +812,14 @@ __device__ __forceinline__ void prefill_tc_body(const Params& p, const CUtensorM
       if (keys < BN) {
         uint8_t* vb = smem_gen + ring_off + (ld_v(n) % nst) * L::KV_BYTES;
         const int first = max(keys, 0);
-        const int chunks = (BN - first) * 8 * HALVES;       // 16-byte chunks to clear
-        for (int idx = lane; idx < chunks; idx += 32) {
-          const int h = idx / ((BN - first) * 8), rem = idx % ((BN - first) * 8);
-          const int key = first + (rem >> 3);
-          *reinterpret_cast<uint4*>(vb + (key >> 3) * L::GROUP_BYTES + h * 1024 + (key & 7) * 128 + ((rem & 7) << 4)) =
-              make_uint4(0, 0, 0, 0);
-        }
+        const int chunks = (BN - first) * 8;                // 16-byte chunks to clear per 64-dim half
+#pragma unroll
+        for (int h = 0; h < HALVES; ++h)
+          for (int idx = lane; idx < chunks; idx += 32) {
+            const int key = first + (idx >> 3);
+            *reinterpret_cast<uint4*>(vb + (key >> 3) * L::GROUP_BYTES + h * 1024 + (key & 7) * 128 + ((idx & 7) << 4)) =
+                make_uint4(0, 0, 0, 0);
+          }
         fence_async_smem();
         __syncwarp();
       }
@@ -652,12 +890,14 @@ prefill_tc_kernel(const Params p, const __grid_constant__ CUtensorMap map_k, con
     dst[1] = __ldg(src + 1);
   }
   const int rows_here = it.new_len * p.G - it.row0;
-  // the two shapes of a CTA are separate instantiations: ring size, load order and the
+  // the three shapes of a CTA are separate instantiations: ring size, load order and the
   // query-tile choice are compile-time constants in the issuing warps' inner loops
   if (rows_here > BM)
-    prefill_tc_body<D, true>(p, map_k, map_v, it);
+    prefill_tc_body<D, 1>(p, map_k, map_v, it);
+  else if (rows_here <= 32)
+    prefill_tc_body<D, 2>(p, map_k, map_v, it);
   else
-    prefill_tc_body<D, false>(p, map_k, map_v, it);
+    prefill_tc_body<D, 0>(p, map_k, map_v, it);
 }
 
 // Merge the KV-chunk partials of split sequences: one warp per (token, head).

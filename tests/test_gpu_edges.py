@@ -253,6 +253,31 @@ def test_many_single_tile_items_beside_long_row_blocks():
     assert np.array_equal(H.torch_to_bits(dw.out), first[0]) and np.array_equal(dw.lse.cpu().numpy(), first[1])
 
 
+@pytest.mark.parametrize("Hq,Hkv,D,cached,new", [
+    (28, 4, 128, [5000, 130, 0, 2047, 900], [1, 4, 3, 1, 2]),        # 7, 28, 21 rows; odd and even tile counts
+    (8, 2, 128, [12000, 1, 127, 128, 255], [8, 8, 7, 1, 8]),         # 32 rows exactly; one key tile; tile edges
+    (4, 4, 64, [3000, 40, 513], [32, 33, 31]),                       # 32 rows / 33 rows: both sides of the boundary
+    (16, 2, 128, [700, 9000], [4, 5]),                               # 32 rows, and 40 rows (the 128-row shape)
+    (32, 8, 128, [16000], [2]),                                      # one long sequence: cut into key chunks
+])
+def test_row_blocks_of_at_most_32_rows(Hq, Hkv, D, cached, new):
+    """Items of at most 32 packed rows (one-token rows of a mixed batch, short `inc`s) run in
+    the CTA shape that holds the rows once per 32-lane quarter and merges eight partial
+    states per row: all rows against the oracle, with and without key chunks, at both head
+    dims, next to items just above the boundary; and the one-call turn (q rotated on load)
+    gives the same bits as the two calls."""
+    efim, H, _custom, _check_turn = _mods()
+    w = _custom(Hq, Hkv, D, cached, new, seed=53)
+    dw, ref = _check_turn(w)
+    two_call = (H.torch_to_bits(dw.out).copy(), dw.lse.cpu().numpy().copy())
+    b = H.DeviceWorkload(w)
+    ws = torch.empty(max(efim.efim_prefill_workspace_bytes(b.cache, b.batch), 256), dtype=torch.uint8, device="cuda")
+    efim.efim_append_prefill_step(b.cache, b.batch, b.rope, b.q, b.k_new, b.v_new, b.out, b.lse, 0.0, ws, b.status)
+    torch.cuda.synchronize()
+    assert int(b.status.item()) == 0
+    assert np.array_equal(H.torch_to_bits(b.out), two_call[0]) and np.array_equal(b.lse.cpu().numpy(), two_call[1])
+
+
 @pytest.mark.parametrize("Hq,Hkv,D", [(8, 2, 128), (4, 4, 64), (7, 1, 128)])
 def test_decode_rows_of_very_different_lengths_in_a_few_chunks(Hq, Hkv, D):
     """A handful of chunks per row: rows that end in the first chunk (their later chunks have
